@@ -1,0 +1,156 @@
+/*
+ * libdab — distribution-aware binarization (DAB-Net, arXiv 1804.02941) inference hot path for
+ * NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no C++ or framework types.
+ *
+ * Vocabulary (paper, Section 4.1): a row W in R^n (a flattened weight filter, n = c*w*h, or an
+ * activation patch in the same element order) is coded as  W~ = alpha*e + beta*(1-e),
+ * e in {0,1}^n, K = e^T e.  The weight side of a contraction carries (e, K_e, alpha, beta), the
+ * activation side (f, K_f, gamma, delta).
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; h_* are HOST pointers.  The
+ *     library allocates and frees no device memory and keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue
+ *     work on that stream and return without synchronising, except where stated.
+ *   - Errors are return codes.  Arguments are validated on the host before anything is
+ *     launched; nothing aborts, traps or throws.  There is no CPU fallback.
+ *   - Packed masks: 32-bit words, element i of a row is bit (i mod 32) of word (i div 32).  A row
+ *     occupies ld words, ld >= ceil(n/32) and ld % 4 == 0, base pointer 16-byte aligned.  Bits
+ *     beyond n and words beyond ceil(n/32) are written as 0 by the producers and must be 0 for
+ *     the consumers.
+ *   - Row length limit: 1 <= n <= DAB_MAX_N.
+ */
+#ifndef DAB_H
+#define DAB_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DAB_MAX_N 16384
+
+typedef enum {
+  DAB_OK = 0,
+  DAB_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad stride or alignment */
+  DAB_ERR_UNSUPPORTED = 2, /* a size beyond a documented limit */
+  DAB_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  DAB_ERR_CUDA = 4         /* a CUDA runtime call or a kernel launch failed */
+} dab_status;
+
+#define DAB_ROW_DEGENERATE 1u /* all values of the row are equal (n == 1 included): K = 0, empty mask, alpha = beta */
+#define DAB_ROW_NONFINITE 2u  /* a NaN or an infinity was seen: K = 0, empty mask, alpha = beta = NaN */
+
+const char* dab_status_string(dab_status s);
+int32_t dab_words_per_row(int32_t n); /* ceil(n/32) */
+int32_t dab_default_ld(int32_t n);    /* dab_words_per_row rounded up to a multiple of 4 words (16 bytes) */
+
+/*
+ * dab_binarize — optimal two-level code of every row (Section 4.1 "Derivation"; Algorithm 1
+ * "Finding an optimal K value"; Section 4.3.1 on treating all filters as one 2-D array).
+ *
+ * For each row: sort, prefix sums P_s, total T, objective D_s = P_s^2/s + (T-P_s)^2/(n-s) over the
+ * splits s = 1..n-1 that fall between two distinct values, maximum with ">=" (the largest s wins
+ * exact ties).  The low partition has mean m_lo = P_s/s, the high one m_hi = (T-P_s)/(n-s).  e marks
+ * the partition whose mean is larger in magnitude (the high one when equal); alpha is that mean,
+ * beta the other.  All of it in fp64; alpha and beta are rounded once to fp32.  -0.0 counts as +0.0.
+ *
+ *   d_values    rows x n fp32, row r at d_values + r*ld_values (ld_values >= n)
+ *   d_K         out, rows int32
+ *   d_alpha     out, rows fp32;  d_beta likewise
+ *   d_mask      out, rows x ld_mask words (see "Packed masks")
+ *   d_row_flags out, rows uint32 of DAB_ROW_* bits; may be NULL
+ * rows == 0 is a no-op returning DAB_OK.
+ */
+dab_status dab_binarize(const float* d_values, int64_t rows, int32_t n, int64_t ld_values, int32_t* d_K,
+                        float* d_alpha, float* d_beta, uint32_t* d_mask, int32_t ld_mask, uint32_t* d_row_flags,
+                        void* stream);
+
+/*
+ * dab_pack — 0/1 bytes to packed words (the mask e of Section 4.1 in the bit layout above; any
+ * non-zero byte counts as 1).
+ *   d_bits  rows x n bytes, row r at d_bits + r*ld_bits (ld_bits >= n)
+ *   d_mask  out, rows x ld_mask words
+ *   d_K     out, rows int32 = number of ones per row; may be NULL
+ */
+dab_status dab_pack(const uint8_t* d_bits, int64_t rows, int32_t n, int64_t ld_bits, uint32_t* d_mask,
+                    int32_t ld_mask, int32_t* d_K, void* stream);
+
+/*
+ * dab_binary_gemm — all dot products between M activation-side rows and N weight-side rows of
+ * two-level codes.  With W~ = alpha e + beta(1-e) (Section 4.1) and X~ = gamma f + delta(1-f), the
+ * forward product of Section 4.3.2 expands over the four 0/1 indicator pairs:
+ *   C[i,j] = alpha_j gamma_i p11 + alpha_j delta_i p10 + beta_j gamma_i p01 + beta_j delta_i p00,
+ *   p11 = popc(e_j & f_i), p10 = K_e - p11, p01 = K_f - p11, p00 = n - K_e - K_f + p11
+ * evaluated in fp64 from the fp32 scalars in exactly that order of terms, rounded once to fp32.
+ *
+ *   d_A, lda, d_KA, d_gamma, d_delta   activation side: M packed rows, their K_f, gamma, delta
+ *   d_B, ldb, d_KB, d_alpha, d_beta    weight side: N packed rows, their K_e, alpha, beta
+ *   d_C, ldc                           out, row-major M x N fp32, row stride ldc >= N
+ *   d_p11, ldp                         out, raw AND-popcounts (int32, row stride ldp >= N); may be NULL
+ */
+dab_status dab_binary_gemm(int64_t M, int64_t N, int32_t n, const uint32_t* d_A, int32_t lda, const int32_t* d_KA,
+                           const float* d_gamma, const float* d_delta, const uint32_t* d_B, int32_t ldb,
+                           const int32_t* d_KB, const float* d_alpha, const float* d_beta, float* d_C, int64_t ldc,
+                           int32_t* d_p11, int64_t ldp, void* stream);
+
+typedef struct {
+  int32_t N, C, H, W;     /* input, NCHW fp32 */
+  int32_t Cout, kh, kw;   /* filters, each flattened in (c, kh, kw) order: n = C*kh*kw */
+  int32_t stride_h, stride_w, pad_h, pad_w;
+} dab_conv_desc;
+
+/* Output extent of a convolution; returns DAB_ERR_INVALID_ARG for an impossible geometry. */
+dab_status dab_conv_output_size(const dab_conv_desc* desc, int32_t* Ho, int32_t* Wo);
+
+/* Bytes of scratch dab_binary_conv needs for this geometry (0 if the descriptor is invalid). */
+size_t dab_binary_conv_workspace(const dab_conv_desc* desc);
+
+/*
+ * dab_binary_conv — the binary forward pass I (*) W~ of Section 4.3.2 with every input patch coded
+ * like a filter: each patch (the C*kh*kw values under one output position, element order (c, kh, kw),
+ * zero padding present as 0.0 values) is binarized as in dab_binarize, then contracted with every
+ * pre-binarized filter as in dab_binary_gemm.  No bias (the paper's binarized layers have none).
+ *
+ *   d_x                          N x C x H x W fp32
+ *   d_wmask, ldw, d_wK, d_walpha, d_wbeta   the filters as written by dab_binarize on [Cout x C*kh*kw]
+ *   d_y                          out, N x Cout x Ho x Wo fp32
+ *   d_workspace, workspace_bytes scratch of at least dab_binary_conv_workspace(desc) bytes, 256-byte aligned
+ * Optional outputs (each may be NULL), patch index p = (img*Ho + ho)*Wo + wo:
+ *   d_pK, d_pgamma, d_pdelta     per-patch K_f, gamma, delta
+ *   d_pmask, ldp                 per-patch packed masks, ldp words apart
+ *   d_pflags                     per-patch DAB_ROW_* bits
+ *   d_p11                        raw AND-popcounts, patches x Cout int32
+ */
+dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                           const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
+                           void* d_workspace, size_t workspace_bytes, int32_t* d_pK, float* d_pgamma,
+                           float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, int32_t* d_p11,
+                           void* stream);
+
+/*
+ * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory: copies h_x
+ * to the device, runs dab_binary_conv, copies the result to h_y, all on `stream`, and returns after
+ * the stream has drained.  Pinned host memory makes the copies asynchronous to other streams.
+ * The scratch must hold dab_binary_conv_host_workspace(desc) bytes (input + output + conv scratch).
+ */
+size_t dab_binary_conv_host_workspace(const dab_conv_desc* desc);
+dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,
+                                const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* h_y,
+                                void* d_workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * dab_popc_probe — measurement aid, not part of the method: runs `iters` rounds of independent
+ * AND + population-count + add chains in every thread of a grid of `blocks` x 256 threads and
+ * writes one word per thread to d_sink (blocks*256 words), so that a caller timing it obtains the
+ * device's achievable rate for the inner operation of dab_binary_gemm.
+ * Word operations executed = blocks * 256 * iters * 16.
+ */
+dab_status dab_popc_probe(uint32_t* d_sink, int32_t blocks, int32_t iters, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

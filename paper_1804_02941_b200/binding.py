@@ -1,0 +1,259 @@
+"""ctypes binding of libdab.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors used as device memory; every step of the method runs inside the
+library's kernels.  If the library has not been built or cannot be loaded, importing the functions
+raises: there is no other implementation to fall back to.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdab.so")
+
+DAB_OK = 0
+DAB_MAX_N = 16384
+ROW_DEGENERATE = 1
+ROW_NONFINITE = 2
+
+EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_binarize", "dab_pack", "dab_binary_gemm",
+           "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binary_conv_host_workspace",
+           "dab_binary_conv_host", "dab_popc_probe")
+
+
+class DabError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("N", "C", "H", "W", "Cout", "kh", "kw", "stride_h", "stride_w", "pad_h", "pad_w")]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libdab.so (raises if it is missing: build it with `python -m paper_1804_02941_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libdab.so not built at %s; run `python -m paper_1804_02941_b200.build`" % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        L.dab_status_string.restype = C.c_char_p
+        L.dab_status_string.argtypes = [C.c_int]
+        L.dab_words_per_row.restype = C.c_int32
+        L.dab_default_ld.restype = C.c_int32
+        L.dab_binary_conv_workspace.restype = C.c_size_t
+        L.dab_binary_conv_host_workspace.restype = C.c_size_t
+        vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int32
+        L.dab_binarize.argtypes = [vp, i64, i32, i64, vp, vp, vp, vp, i32, vp, vp]
+        L.dab_pack.argtypes = [vp, i64, i32, i64, vp, i32, vp, vp]
+        L.dab_binary_gemm.argtypes = [i64, i64, i32, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, i64, vp, i64, vp]
+        L.dab_conv_output_size.argtypes = [vp, vp, vp]
+        L.dab_binary_conv_workspace.argtypes = [vp]
+        L.dab_binary_conv_host_workspace.argtypes = [vp]
+        L.dab_binary_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp, vp, vp, vp, i32, vp, vp, vp]
+        L.dab_binary_conv_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().dab_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != DAB_OK:
+        raise DabError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _dev(t, dtype, name):
+    if not isinstance(t, torch.Tensor) or not t.is_cuda or t.dtype != dtype:
+        raise TypeError("%s must be a CUDA tensor of dtype %s" % (name, dtype))
+    return t
+
+
+def dab_words_per_row(n: int) -> int:
+    return int(lib().dab_words_per_row(C.c_int32(n)))
+
+
+def dab_default_ld(n: int) -> int:
+    return int(lib().dab_default_ld(C.c_int32(n)))
+
+
+@dataclass
+class Coded:
+    """Two-level codes of a batch of rows, as device tensors."""
+    mask: torch.Tensor    # rows x ld int32 (bit pattern of the uint32 words)
+    K: torch.Tensor       # rows int32
+    alpha: torch.Tensor   # rows fp32
+    beta: torch.Tensor    # rows fp32
+    flags: torch.Tensor   # rows int32 (ROW_* bits)
+    n: int
+
+    @property
+    def ld(self) -> int:
+        return self.mask.shape[1]
+
+
+def dab_binarize(values: torch.Tensor, ld_mask: int | None = None, stream=None) -> Coded:
+    """rows x n fp32 (row stride = values.stride(0)) -> K, alpha, beta, packed mask, flags."""
+    _dev(values, torch.float32, "values")
+    if values.dim() != 2 or values.stride(1) != 1:
+        raise ValueError("values must be 2-D with unit inner stride")
+    rows, n = values.shape
+    ld = dab_default_ld(n) if ld_mask is None else ld_mask
+    dev = values.device
+    out = Coded(torch.empty((rows, ld), dtype=torch.int32, device=dev), torch.empty(rows, dtype=torch.int32, device=dev),
+                torch.empty(rows, dtype=torch.float32, device=dev), torch.empty(rows, dtype=torch.float32, device=dev),
+                torch.empty(rows, dtype=torch.int32, device=dev), n)
+    ldv = values.stride(0) if rows > 1 else max(n, values.stride(0))
+    st = lib().dab_binarize(_ptr(values), rows, n, ldv, _ptr(out.K), _ptr(out.alpha), _ptr(out.beta), _ptr(out.mask),
+                            ld, _ptr(out.flags), _stream(stream))
+    _check(st, "dab_binarize")
+    return out
+
+
+def dab_binarize_into(values, K, alpha, beta, mask, flags=None, stream=None) -> None:
+    """Same call with caller-provided outputs (no allocation)."""
+    rows, n = values.shape
+    ldv = values.stride(0) if rows > 1 else max(n, values.stride(0))
+    st = lib().dab_binarize(_ptr(values), rows, n, ldv, _ptr(K), _ptr(alpha), _ptr(beta), _ptr(mask), mask.stride(0),
+                            _ptr(flags), _stream(stream))
+    _check(st, "dab_binarize")
+
+
+def dab_pack(bits: torch.Tensor, ld_mask: int | None = None, stream=None):
+    """rows x n uint8 (0/1) -> (rows x ld int32 words, K int32)."""
+    _dev(bits, torch.uint8, "bits")
+    if bits.dim() != 2 or bits.stride(1) != 1:
+        raise ValueError("bits must be 2-D with unit inner stride")
+    rows, n = bits.shape
+    ld = dab_default_ld(n) if ld_mask is None else ld_mask
+    mask = torch.empty((rows, ld), dtype=torch.int32, device=bits.device)
+    K = torch.empty(rows, dtype=torch.int32, device=bits.device)
+    ldb = bits.stride(0) if rows > 1 else max(n, bits.stride(0))
+    _check(lib().dab_pack(_ptr(bits), rows, n, ldb, _ptr(mask), ld, _ptr(K), _stream(stream)), "dab_pack")
+    return mask, K
+
+
+def dab_binary_gemm(a: Coded, b: Coded, want_p11: bool = False, out: torch.Tensor | None = None, stream=None):
+    """C[i,j] = coded row i of `a` (activation side) . coded row j of `b` (weight side); M x N fp32."""
+    if a.n != b.n:
+        raise ValueError("row lengths differ")
+    M, N = a.mask.shape[0], b.mask.shape[0]
+    dev = a.mask.device
+    Cm = torch.empty((M, N), dtype=torch.float32, device=dev) if out is None else out
+    p11 = torch.empty((M, N), dtype=torch.int32, device=dev) if want_p11 else None
+    st = lib().dab_binary_gemm(M, N, a.n, _ptr(a.mask), a.ld, _ptr(a.K), _ptr(a.alpha), _ptr(a.beta), _ptr(b.mask),
+                               b.ld, _ptr(b.K), _ptr(b.alpha), _ptr(b.beta), _ptr(Cm), Cm.stride(0) if M > 1 else max(N, 1),
+                               _ptr(p11), N, _stream(stream))
+    _check(st, "dab_binary_gemm")
+    return (Cm, p11) if want_p11 else Cm
+
+
+def make_desc(x_shape, Cout, kh, kw, stride=(1, 1), pad=(0, 0)) -> ConvDesc:
+    N, Cc, H, W = x_shape
+    return ConvDesc(N, Cc, H, W, Cout, kh, kw, stride[0], stride[1], pad[0], pad[1])
+
+
+def dab_conv_output_size(desc: ConvDesc):
+    ho, wo = C.c_int32(), C.c_int32()
+    _check(lib().dab_conv_output_size(C.byref(desc), C.byref(ho), C.byref(wo)), "dab_conv_output_size")
+    return ho.value, wo.value
+
+
+def dab_binary_conv_workspace(desc: ConvDesc) -> int:
+    return int(lib().dab_binary_conv_workspace(C.byref(desc)))
+
+
+def dab_binary_conv_host_workspace(desc: ConvDesc) -> int:
+    return int(lib().dab_binary_conv_host_workspace(C.byref(desc)))
+
+
+@dataclass
+class ConvDetails:
+    pK: torch.Tensor
+    pgamma: torch.Tensor
+    pdelta: torch.Tensor
+    pmask: torch.Tensor
+    pflags: torch.Tensor
+    p11: torch.Tensor
+
+
+def dab_binary_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0), details: bool = False,
+                    y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None):
+    """x: N x C x H x W fp32 (contiguous); w: filters coded by dab_binarize on [Cout x C*kh*kw] -> y NCHW fp32."""
+    _dev(x, torch.float32, "x")
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous NCHW")
+    Cout = w.mask.shape[0]
+    desc = make_desc(tuple(x.shape), Cout, kh, kw, stride, pad)
+    if w.n != x.shape[1] * kh * kw:
+        raise ValueError("filter length does not match C*kh*kw")
+    Ho, Wo = dab_conv_output_size(desc)
+    dev = x.device
+    if y is None:
+        y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=dev)
+    need = dab_binary_conv_workspace(desc)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    det = None
+    if details:
+        P = x.shape[0] * Ho * Wo
+        det = ConvDetails(torch.empty(P, dtype=torch.int32, device=dev), torch.empty(P, dtype=torch.float32, device=dev),
+                          torch.empty(P, dtype=torch.float32, device=dev),
+                          torch.empty((P, dab_default_ld(w.n)), dtype=torch.int32, device=dev),
+                          torch.empty(P, dtype=torch.int32, device=dev),
+                          torch.empty((P, Cout), dtype=torch.int32, device=dev))
+    st = lib().dab_binary_conv(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha), _ptr(w.beta),
+                               _ptr(y), _ptr(workspace), workspace.numel(),
+                               _ptr(det.pK) if det else None, _ptr(det.pgamma) if det else None,
+                               _ptr(det.pdelta) if det else None, _ptr(det.pmask) if det else None,
+                               det.pmask.shape[1] if det else 0, _ptr(det.pflags) if det else None,
+                               _ptr(det.p11) if det else None, _stream(stream))
+    _check(st, "dab_binary_conv")
+    return (y, det) if details else y
+
+
+def dab_binary_conv_host(x_host: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
+                         y_host: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None):
+    """Host tensors in and out (pinned memory recommended); the library does the copies. Synchronous."""
+    if x_host.is_cuda or x_host.dtype != torch.float32 or not x_host.is_contiguous():
+        raise TypeError("x_host must be a contiguous fp32 host tensor")
+    Cout = w.mask.shape[0]
+    desc = make_desc(tuple(x_host.shape), Cout, kh, kw, stride, pad)
+    Ho, Wo = dab_conv_output_size(desc)
+    if y_host is None:
+        y_host = torch.empty((x_host.shape[0], Cout, Ho, Wo), dtype=torch.float32).pin_memory()
+    need = dab_binary_conv_host_workspace(desc)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=w.mask.device)
+    st = lib().dab_binary_conv_host(C.byref(desc), C.c_void_p(x_host.data_ptr()), _ptr(w.mask), w.ld, _ptr(w.K),
+                                    _ptr(w.alpha), _ptr(w.beta), C.c_void_p(y_host.data_ptr()), _ptr(workspace),
+                                    workspace.numel(), _stream(stream))
+    _check(st, "dab_binary_conv_host")
+    return y_host
+
+
+def dab_popc_probe(blocks: int, iters: int, sink: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    if sink is None:
+        sink = torch.empty(blocks * 256, dtype=torch.int32, device="cuda")
+    _check(lib().dab_popc_probe(_ptr(sink), blocks, iters, _stream(stream)), "dab_popc_probe")
+    return sink

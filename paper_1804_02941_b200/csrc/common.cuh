@@ -1,0 +1,72 @@
+// Shared device helpers and internal launch declarations of libdab (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dab.h"
+
+namespace dab {
+
+constexpr uint32_t kPadKey = 0xFFFFFFFFu;
+
+// Monotone map fp32 -> uint32: a < b  <=>  key(a) < key(b); -0.0 and +0.0 share one key.
+__device__ __forceinline__ uint32_t order_key(float x) {
+  uint32_t b = __float_as_uint(x);
+  if (b == 0x80000000u) b = 0u;
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ float key_value(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+__device__ __forceinline__ bool is_nonfinite(float x) {
+  return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u;
+}
+
+// Objective of Algorithm 1 for a low partition of size s with sum P, row total T, row length n.
+// Every operation rounds on its own (no fused multiply-add), in this order.
+__device__ __forceinline__ double objective(double P, double T, int s, int n) {
+  double Q = __dsub_rn(T, P);
+  return __dadd_rn(__ddiv_rn(__dmul_rn(P, P), (double)s), __ddiv_rn(__dmul_rn(Q, Q), (double)(n - s)));
+}
+
+// Where an output element (row i of the activation side, column j of the weight side) is stored:
+//   offset = (i / inner) * outer_stride + (i % inner) * row_stride + j * col_stride
+// Row-major M x N: inner = M (never wraps), row_stride = ldc, col_stride = 1.
+// NCHW conv output: inner = Ho*Wo, outer_stride = Cout*Ho*Wo, row_stride = 1, col_stride = Ho*Wo.
+struct OutMap {
+  int64_t inner, outer_stride, row_stride, col_stride;
+};
+
+struct GemmArgs {
+  int64_t M, N;
+  int32_t n, words;  // words = ceil(n/32) rounded up to a multiple of 4 (<= lda, ldb)
+  const uint32_t* A;
+  int32_t lda;
+  const int32_t* KA;
+  const float* gamma;
+  const float* delta;
+  const uint32_t* B;
+  int32_t ldb;
+  const int32_t* KB;
+  const float* alpha;
+  const float* beta;
+  float* C;
+  OutMap map;
+  int32_t* p11;
+  int64_t ldp;
+};
+
+cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
+                            float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
+                            cudaStream_t stream);
+cudaError_t launch_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld_bits, uint32_t* mask,
+                        int32_t ld_mask, int32_t* K, cudaStream_t stream);
+cudaError_t launch_gemm(const GemmArgs& args, bool lanes_along_rows, cudaStream_t stream);
+cudaError_t launch_im2col(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int64_t patch_begin,
+                          int64_t patch_count, float* patches, cudaStream_t stream);
+cudaError_t launch_popc_probe(uint32_t* sink, int32_t blocks, int32_t iters, cudaStream_t stream);
+
+}  // namespace dab
