@@ -10,11 +10,10 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline dab_status from_cuda(cudaError_t e) { return e == cudaSuccess ? DAB_OK : DAB_ERR_CUDA; }
 
 constexpr size_t kAlign = 256;
-constexpr size_t kPatchChunkBytes = size_t(256) << 20;  // patch values staged per pass of the general conv path
 
 struct ConvGeom {
   int32_t Ho, Wo, n, ld;
-  int64_t patches, chunk;
+  int64_t patches;
 };
 
 bool conv_geom(const dab_conv_desc* d, ConvGeom* g) {
@@ -30,14 +29,11 @@ bool conv_geom(const dab_conv_desc* d, ConvGeom* g) {
   g->n = (int32_t)n;
   g->ld = dab_default_ld((int32_t)n);
   g->patches = (int64_t)d->N * g->Ho * g->Wo;
-  int64_t chunk = (int64_t)(kPatchChunkBytes / (sizeof(float) * (size_t)n));
-  if (chunk < 1) chunk = 1;
-  g->chunk = chunk < g->patches ? chunk : g->patches;
   return true;
 }
 
 struct ConvScratch {
-  size_t off_K, off_gamma, off_delta, off_flags, off_mask, off_patches, total;
+  size_t off_K, off_gamma, off_delta, off_mask, total;
 };
 
 ConvScratch conv_scratch(const ConvGeom& g) {
@@ -46,9 +42,7 @@ ConvScratch conv_scratch(const ConvGeom& g) {
   s.off_K = o;       o += round_up(P * sizeof(int32_t), kAlign);
   s.off_gamma = o;   o += round_up(P * sizeof(float), kAlign);
   s.off_delta = o;   o += round_up(P * sizeof(float), kAlign);
-  s.off_flags = o;   o += round_up(P * sizeof(uint32_t), kAlign);
   s.off_mask = o;    o += round_up(P * (size_t)g.ld * sizeof(uint32_t), kAlign);
-  s.off_patches = o; o += round_up((size_t)g.chunk * (size_t)g.n * sizeof(float), kAlign);
   s.total = o;
   return s;
 }
@@ -152,18 +146,11 @@ dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const ui
   int32_t* pK = d_pK ? d_pK : reinterpret_cast<int32_t*>(ws + sc.off_K);
   float* pg = d_pgamma ? d_pgamma : reinterpret_cast<float*>(ws + sc.off_gamma);
   float* pd = d_pdelta ? d_pdelta : reinterpret_cast<float*>(ws + sc.off_delta);
-  uint32_t* pf = d_pflags ? d_pflags : reinterpret_cast<uint32_t*>(ws + sc.off_flags);
   uint32_t* pm = d_pmask ? d_pmask : reinterpret_cast<uint32_t*>(ws + sc.off_mask);
   int32_t ldm = d_pmask ? ldp : g.ld;
-  float* patches = reinterpret_cast<float*>(ws + sc.off_patches);
 
-  for (int64_t p0 = 0; p0 < g.patches; p0 += g.chunk) {
-    int64_t cnt = g.patches - p0 < g.chunk ? g.patches - p0 : g.chunk;
-    cudaError_t e = launch_im2col(*desc, g.Ho, g.Wo, d_x, p0, cnt, patches, st);
-    if (e != cudaSuccess) return DAB_ERR_CUDA;
-    e = launch_binarize(patches, cnt, g.n, g.n, pK + p0, pg + p0, pd + p0, pm + p0 * ldm, ldm, pf + p0, st);
-    if (e != cudaSuccess) return DAB_ERR_CUDA;
-  }
+  if (launch_binarize_patches(*desc, g.Ho, g.Wo, d_x, pK, pg, pd, pm, ldm, d_pflags, st) != cudaSuccess)
+    return DAB_ERR_CUDA;
 
   GemmArgs a;
   a.M = g.patches; a.N = desc->Cout; a.n = g.n; a.words = (dab_words_per_row(g.n) + 3) / 4 * 4;

@@ -1,203 +1,243 @@
-// dab_binarize: one CTA per row.  Sort the row's order-preserving keys in shared memory, scan the
-// sorted values in fp64, evaluate the objective of Algorithm 1 at every split between distinct
-// values, reduce to the arg-max under the tie rule, then write K, alpha, beta and the packed mask.
-#include "common.cuh"
+// dab_binarize (rows of a matrix) and the patch coder of dab_binary_conv (patches of an NCHW tensor).
+// Both drive the same group-of-warps row coder (rowcode.cuh); they differ in where a row's values come from
+// and where the results go.
+#include "rowcode.cuh"
 
 namespace dab {
 
-struct Best {
-  double D;
-  double P;
-  int s;
-};
-
-__device__ __forceinline__ bool better(const Best& a, const Best& b) {  // is a preferred over b
-  return a.D > b.D || (a.D == b.D && a.s > b.s);
-}
-
-__device__ __forceinline__ Best shfl_down_best(const Best& v, int off) {
-  Best r;
-  r.D = __shfl_down_sync(0xFFFFFFFFu, v.D, off);
-  r.P = __shfl_down_sync(0xFFFFFFFFu, v.P, off);
-  r.s = __shfl_down_sync(0xFFFFFFFFu, v.s, off);
-  return r;
-}
-
-template <int NPAD, int THREADS>
-__global__ void __launch_bounds__(THREADS) binarize_rows_kernel(const float* __restrict__ values, int64_t rows,
-                                                                int32_t n, int64_t ld_values,
-                                                                int32_t* __restrict__ K_out,
-                                                                float* __restrict__ alpha_out,
-                                                                float* __restrict__ beta_out,
-                                                                uint32_t* __restrict__ mask_out, int32_t ld_mask,
-                                                                uint32_t* __restrict__ flags_out) {
-  constexpr int L = NPAD / THREADS;  // sorted positions owned by one thread in the scan
-  constexpr int WARPS = THREADS / 32;
-  static_assert(NPAD % THREADS == 0 && THREADS % 32 == 0, "shape");
-  extern __shared__ uint32_t keys[];  // NPAD keys
-  __shared__ double warp_sum[WARPS];
-  __shared__ Best warp_best[WARPS];
-  __shared__ uint32_t s_tkey;
-  __shared__ int s_mode;  // 0: e = [w >= t], 1: e = [w < t], 2: empty mask
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
-    const float* v = values + row * ld_values;
-    uint32_t* mrow = mask_out + row * (int64_t)ld_mask;
-
-    int bad = 0;
-    for (int i = tid; i < NPAD; i += THREADS) {
-      uint32_t k = kPadKey;
-      if (i < n) {
-        float x = v[i];
-        bad |= is_nonfinite(x);
-        k = order_key(x);
-      }
-      keys[i] = k;
-    }
-    bad = __syncthreads_or(bad);
-
-    if (!bad) {
-      // Bitonic sort, ascending; the pad keys end up behind the n real ones.
-      for (int k = 2; k <= NPAD; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-          for (int t = tid; t < NPAD / 2; t += THREADS) {
-            int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-            int p = i | j;
-            uint32_t a = keys[i], b = keys[p];
-            bool up = (i & k) == 0;
-            if ((a > b) == up) {
-              keys[i] = b;
-              keys[p] = a;
-            }
-          }
-          __syncthreads();
-        }
-      }
-    }
-
-    const bool constant = !bad && keys[0] == keys[n - 1];
-
-    if (!bad && !constant) {
-      // fp64 sum of the thread's run of sorted values, then an exclusive scan across the CTA.
-      const int base = tid * L;
-      double local = 0.0;
-#pragma unroll 4
-      for (int q = 0; q < L; ++q) {
-        int pos = base + q;
-        if (pos < n) local = __dadd_rn(local, (double)key_value(keys[pos]));
-      }
-      double incl = local;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        double o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-        if (lane >= off) incl = __dadd_rn(incl, o);
-      }
-      if (lane == 31) warp_sum[warp] = incl;
-      __syncthreads();
-      double before = 0.0, T = 0.0;
-#pragma unroll
-      for (int w = 0; w < WARPS; ++w) {
-        double ws = warp_sum[w];
-        if (w < warp) before = __dadd_rn(before, ws);
-        T = __dadd_rn(T, ws);
-      }
-      double P = __dadd_rn(before, __dsub_rn(incl, local));
-
-      Best best;
-      best.D = -1.0;
-      best.P = 0.0;
-      best.s = 0;
-      for (int q = 0; q < L; ++q) {
-        int pos = base + q;
-        if (pos >= n - 1) break;
-        uint32_t kc = keys[pos];
-        P = __dadd_rn(P, (double)key_value(kc));
-        if (kc == keys[pos + 1]) continue;  // never split a run of equal values
-        int s = pos + 1;
-        double D = objective(P, T, s, n);
-        if (D >= best.D) {  // ascending s: ">=" keeps the largest s among equal objectives
-          best.D = D;
-          best.P = P;
-          best.s = s;
-        }
-      }
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        Best o = shfl_down_best(best, off);
-        if (better(o, best)) best = o;
-      }
-      if (lane == 0) warp_best[warp] = best;
-      __syncthreads();
-      if (tid == 0) {
-        for (int w = 1; w < WARPS; ++w)
-          if (better(warp_best[w], best)) best = warp_best[w];
-        double m_lo = __ddiv_rn(best.P, (double)best.s);
-        double m_hi = __ddiv_rn(__dsub_rn(T, best.P), (double)(n - best.s));
-        bool low_side = fabs(m_lo) > fabs(m_hi);  // e marks the partition whose mean is larger in magnitude
-        s_tkey = keys[best.s];                    // smallest value of the high partition
-        s_mode = low_side ? 1 : 0;
-        K_out[row] = low_side ? best.s : n - best.s;
-        alpha_out[row] = (float)(low_side ? m_lo : m_hi);
-        beta_out[row] = (float)(low_side ? m_hi : m_lo);
-        if (flags_out) flags_out[row] = 0u;
-      }
-    } else if (tid == 0) {
-      s_mode = 2;
-      s_tkey = 0u;
-      K_out[row] = 0;
-      float c = bad ? __uint_as_float(0x7FC00000u) : key_value(keys[0]);
-      alpha_out[row] = c;
-      beta_out[row] = c;
-      if (flags_out) flags_out[row] = bad ? DAB_ROW_NONFINITE : DAB_ROW_DEGENERATE;
-    }
-    __syncthreads();
-
-    const uint32_t tkey = s_tkey;
-    const int mode = s_mode;
-    for (int w = warp; w < ld_mask; w += WARPS) {
-      int i = w * 32 + lane;
+// Writes the packed mask of one row: the group's warps take 32-word batches; lane t keeps word t of a batch so
+// that a batch is stored with one coalesced write.  Words between ceil(n/32) and ld are written as 0.
+template <int W, typename Value>
+__device__ __forceinline__ void group_write_mask(Value value, int n, int ld, const RowResult& res, int tig,
+                                                 uint32_t* __restrict__ out) {
+  const int lane = tig & 31, warp = tig >> 5;
+  const bool flip = res.mode == 1;
+  for (int w0 = warp * 32; w0 < ld; w0 += 32 * W) {
+    uint32_t mine = 0;
+    const int wend = min(32, ld - w0);
+    for (int t = 0; t < wend; ++t) {
+      int i = (w0 + t) * 32 + lane;
       bool bit = false;
-      if (mode != 2 && i < n) bit = (order_key(v[i]) >= tkey) != (mode == 1);
+      if (res.mode != 2 && i < n) bit = (order_key(value(i)) >= res.tkey) != flip;
       uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
-      if (lane == 0) mrow[w] = word;
+      if (lane == t) mine = word;
     }
-    __syncthreads();  // keys and the broadcast slots are reused by the next row
+    if (lane < wend) out[w0 + lane] = mine;
   }
 }
 
-template <int NPAD, int THREADS>
-static cudaError_t launch_one(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
-                              float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                              cudaStream_t stream) {
-  auto kern = binarize_rows_kernel<NPAD, THREADS>;
-  size_t smem = sizeof(uint32_t) * NPAD;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+__host__ __device__ inline int scratch_words_for(int n, int W) {
+  int cap = 128 * W;
+  while (cap < n) cap <<= 1;
+  return cap + (cap >> 5) + 1;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Rows of a matrix.  A CTA of WARPS warps holds WARPS/W groups; each group walks over rows.
+// ---------------------------------------------------------------------------------------------------------
+template <int W, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) binarize_rows_kernel(const float* __restrict__ values, int64_t rows,
+                                                                   int32_t n, int64_t ld_values,
+                                                                   int32_t* __restrict__ K_out,
+                                                                   float* __restrict__ alpha_out,
+                                                                   float* __restrict__ beta_out,
+                                                                   uint32_t* __restrict__ mask_out, int32_t ld_mask,
+                                                                   uint32_t* __restrict__ flags_out,
+                                                                   int scratch_words) {
+  constexpr int G = WARPS / W;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  GroupShared* gs_all = reinterpret_cast<GroupShared*>(smem_raw);
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(smem_raw + sizeof(GroupShared) * G);
+
+  const int group = threadIdx.x / (32 * W);
+  const int tig = threadIdx.x % (32 * W);
+  GroupShared* gs = gs_all + group;
+  uint32_t* scratch = scratch_all + (size_t)group * scratch_words;
+  const int bar_id = 1 + group;
+
+  for (int64_t row = (int64_t)blockIdx.x * G + group; row < rows; row += (int64_t)gridDim.x * G) {
+    const float* v = values + row * ld_values;
+    auto value = [v](int i) { return __ldg(v + i); };
+    group_code_row<W>(value, n, tig, scratch, gs, bar_id);
+    const RowResult res = gs->result;
+    if (tig == 0) {
+      K_out[row] = res.K;
+      alpha_out[row] = res.alpha;
+      beta_out[row] = res.beta;
+      if (flags_out) flags_out[row] = res.flags;
+    }
+    group_write_mask<W>(value, n, ld_mask, res, tig, mask_out + row * (int64_t)ld_mask);
+    group_barrier(bar_id, 32 * W);  // gs->result is overwritten by the next row
   }
-  int64_t grid = rows < (int64_t)(1 << 20) ? rows : (int64_t)(1 << 20);
-  kern<<<(unsigned)grid, THREADS, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags);
+}
+
+template <int W, int WARPS>
+static cudaError_t launch_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
+                               float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
+                               cudaStream_t stream) {
+  constexpr int G = WARPS / W;
+  auto kern = binarize_rows_kernel<W, WARPS>;
+  int sw = scratch_words_for(n, W);
+  size_t smem = sizeof(GroupShared) * G + sizeof(uint32_t) * (size_t)sw * G;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int64_t blocks = (rows + G - 1) / G;
+  const int64_t cap = 148 * 16;
+  if (blocks > cap) blocks = cap;
+  kern<<<(unsigned)blocks, WARPS * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask,
+                                                       flags, sw);
   return cudaGetLastError();
 }
 
 cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                             float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
                             cudaStream_t stream) {
-#define DAB_CASE(NP, TH) \
-  if (n <= NP) return launch_one<NP, TH>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream)
-  DAB_CASE(64, 32);
-  DAB_CASE(128, 64);
-  DAB_CASE(256, 64);
-  DAB_CASE(512, 128);
-  DAB_CASE(1024, 128);
-  DAB_CASE(2048, 256);
-  DAB_CASE(4096, 256);
-  DAB_CASE(8192, 512);
-  DAB_CASE(16384, 512);
-#undef DAB_CASE
-  return cudaErrorInvalidValue;
+#define DAB_ROWS(Wv, WARPSv) \
+  return launch_rows<Wv, WARPSv>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream)
+  if (n <= 1024) DAB_ROWS(1, 8);
+  if (n <= 2048) DAB_ROWS(2, 8);
+  if (n <= 4096) DAB_ROWS(4, 8);
+  if (n <= 8192) DAB_ROWS(8, 8);
+  DAB_ROWS(16, 16);
+#undef DAB_ROWS
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Patches of an NCHW tensor.  A CTA stages the input region under a tile of TH x TW output positions (all
+// channels, zero padding filled in) in shared memory, then its groups code the tile's patches one by one.
+// Element i of a patch, i = (c*kh + r)*kw + s, sits at tile offset off[i] + patch origin.
+// ---------------------------------------------------------------------------------------------------------
+struct PatchArgs {
+  dab_conv_desc d;
+  int32_t Ho, Wo, n;
+  int32_t TH, TW;          // output positions per tile
+  int32_t in_h, in_w;      // staged rows/columns per channel: (TH-1)*stride_h + kh, (TW-1)*stride_w + kw
+  int32_t pitch;           // words per staged row (>= in_w)
+  int32_t tiles_h, tiles_w;
+  int32_t scratch_words;
+  const float* x;
+  int32_t* pK;
+  float* pgamma;
+  float* pdelta;
+  uint32_t* pflags;        // may be null
+  uint32_t* pmask;
+  int32_t ldp;
+};
+
+template <int W, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) binarize_patches_kernel(const PatchArgs a) {
+  constexpr int G = WARPS / W;
+  constexpr int THREADS = WARPS * 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  GroupShared* gs_all = reinterpret_cast<GroupShared*>(smem_raw);
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(smem_raw + sizeof(GroupShared) * G);
+  float* tile = reinterpret_cast<float*>(scratch_all + (size_t)G * a.scratch_words);
+  const int ch_words = a.in_h * a.pitch;
+  uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
+
+  const int group = threadIdx.x / (32 * W);
+  const int tig = threadIdx.x % (32 * W);
+  GroupShared* gs = gs_all + group;
+  uint32_t* scratch = scratch_all + (size_t)group * a.scratch_words;
+  const int bar_id = 1 + group;
+
+  // element offsets inside the tile (same for every patch)
+  const int khw = a.d.kh * a.d.kw;
+  for (int i = threadIdx.x; i < a.n; i += THREADS) {
+    int c = i / khw, rs = i % khw;
+    off[i] = (uint16_t)(c * ch_words + (rs / a.d.kw) * a.pitch + (rs % a.d.kw));
+  }
+
+  const int64_t tiles_per_img = (int64_t)a.tiles_h * a.tiles_w;
+  const int64_t total_tiles = tiles_per_img * a.d.N;
+  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+    const int img = (int)(tile_id / tiles_per_img);
+    const int trem = (int)(tile_id % tiles_per_img);
+    const int ho0 = (trem / a.tiles_w) * a.TH, wo0 = (trem % a.tiles_w) * a.TW;
+    const int h0 = ho0 * a.d.stride_h - a.d.pad_h, w0 = wo0 * a.d.stride_w - a.d.pad_w;
+
+    __syncthreads();  // the previous tile is no longer read
+    const float* ximg = a.x + (int64_t)img * a.d.C * a.d.H * a.d.W;
+    const int per_ch = a.in_h * a.in_w;
+    for (int idx = threadIdx.x; idx < a.d.C * per_ch; idx += THREADS) {
+      int c = idx / per_ch, rem = idx % per_ch;
+      int r = rem / a.in_w, s = rem % a.in_w;
+      int h = h0 + r, w = w0 + s;
+      float v = 0.0f;
+      if (h >= 0 && h < a.d.H && w >= 0 && w < a.d.W) v = __ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w);
+      tile[c * ch_words + r * a.pitch + s] = v;
+    }
+    __syncthreads();
+
+    const int th = min(a.TH, a.Ho - ho0), tw = min(a.TW, a.Wo - wo0);
+    for (int p = group; p < th * tw; p += G) {
+      const int lh = p / tw, lw = p % tw;
+      const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+      auto value = [origin, off](int i) { return origin[off[i]]; };
+      group_code_row<W>(value, a.n, tig, scratch, gs, bar_id);
+      const RowResult res = gs->result;
+      const int64_t pi = ((int64_t)img * a.Ho + (ho0 + lh)) * a.Wo + (wo0 + lw);
+      if (tig == 0) {
+        a.pK[pi] = res.K;
+        a.pgamma[pi] = res.alpha;
+        a.pdelta[pi] = res.beta;
+        if (a.pflags) a.pflags[pi] = res.flags;
+      }
+      group_write_mask<W>(value, a.n, a.ldp, res, tig, a.pmask + pi * (int64_t)a.ldp);
+      group_barrier(bar_id, 32 * W);
+    }
+  }
+}
+
+// Picks the tile: the largest of a few shapes whose staged input fits the shared-memory budget.
+static void choose_tile(const dab_conv_desc& d, int Ho, int Wo, size_t budget_bytes, PatchArgs* a) {
+  static const int shapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
+  for (auto& sh : shapes) {
+    int TH = sh[0] < Ho ? sh[0] : Ho, TW = sh[1] < Wo ? sh[1] : Wo;
+    int in_h = (TH - 1) * d.stride_h + d.kh, in_w = (TW - 1) * d.stride_w + d.kw;
+    int pitch = in_w | 1;  // odd pitch spreads the rows of a patch over the banks
+    size_t bytes = (size_t)d.C * in_h * pitch * sizeof(float);
+    if (bytes <= budget_bytes || (TH == 1 && TW == 1)) {
+      a->TH = TH; a->TW = TW; a->in_h = in_h; a->in_w = in_w; a->pitch = pitch;
+      a->tiles_h = (Ho + TH - 1) / TH; a->tiles_w = (Wo + TW - 1) / TW;
+      return;
+    }
+  }
+}
+
+template <int W, int WARPS>
+static cudaError_t launch_patches_t(PatchArgs& a, cudaStream_t stream) {
+  constexpr int G = WARPS / W;
+  auto kern = binarize_patches_kernel<W, WARPS>;
+  a.scratch_words = scratch_words_for(a.n, W);
+  size_t fixed = sizeof(GroupShared) * G + sizeof(uint32_t) * (size_t)a.scratch_words * G + sizeof(uint16_t) * a.n + 16;
+  const size_t limit = 200 * 1024;
+  size_t budget = limit > fixed ? limit - fixed : 0;
+  if (budget > 72 * 1024) budget = 72 * 1024;  // leave room for more than one CTA per SM when the tile is small
+  choose_tile(a.d, a.Ho, a.Wo, budget, &a);
+  size_t tile_bytes = (size_t)a.d.C * a.in_h * a.pitch * sizeof(float);
+  if ((size_t)a.d.C * a.in_h * a.pitch > 65535) return cudaErrorInvalidValue;  // offsets are 16-bit
+  size_t smem = fixed + tile_bytes;
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int64_t tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  int64_t blocks = tiles < 148 * 8 ? tiles : 148 * 8;
+  kern<<<(unsigned)blocks, WARPS * 32, smem, stream>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
+                                    float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
+                                    cudaStream_t stream) {
+  PatchArgs a;
+  a.d = d; a.Ho = Ho; a.Wo = Wo; a.n = d.C * d.kh * d.kw;
+  a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
+  if (a.n <= 1024) return launch_patches_t<1, 8>(a, stream);
+  if (a.n <= 2048) return launch_patches_t<2, 8>(a, stream);
+  if (a.n <= 4096) return launch_patches_t<4, 8>(a, stream);
+  if (a.n <= 8192) return launch_patches_t<8, 8>(a, stream);
+  return launch_patches_t<16, 16>(a, stream);
 }
 
 }  // namespace dab
