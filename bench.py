@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the DAB-Net inference hot path on B200.
+
+A step is one pass of the whole path over one batch: for each of the 16 binarized 3x3 convolutions of the
+ResNet-18-shaped stack (batch 256), binarize the filters, binarize every input patch, contract the packed
+masks with the rescale fused in.  Every layer gets its own synthetic post-ReLU input (60 % exact zeros).
+Prints ONE JSON line.  `--impl reference` times the CPU checker on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "binary_conv_tops_equiv"
+UNIT = "TOPS-equiv (2*M*N*n binary ops per second / 1e12)"
+L2_BYTES = 126 * 1024 * 1024
+POPC_PER_CLK_PER_SM = 16          # integer population counts per clock per SM
+SM_COUNT = 148
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="dab", choices=["dab", "reference"])
+    ap.add_argument("--batch", type=int, default=256, help="images per step and per GPU (256 = the named workload)")
+    ap.add_argument("--dense", action="store_true", help="N(0,1) inputs without zeros instead of post-ReLU inputs")
+    ap.add_argument("--layers", default="", help="comma-separated layer names (e.g. l1_0,l4_1) to run a subset; "
+                    "the default is the whole workload")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample-batch", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)", float(d.get("sm_max_mhz", 1965.0))
+    return 6650.0, "fallback (earlier measurement on this pool)", 1965.0
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+# ------------------------------------------------------------------------------------------------------------
+# CPU checker timing (the reference arm and the cpu_baseline leg)
+# ------------------------------------------------------------------------------------------------------------
+def oracle_pass(layers, inputs, weights):
+    """One pass of the checker over the sample; returns (seconds, binary ops)."""
+    import oracle
+    t0 = time.perf_counter()
+    ops = 0
+    for L, x, w in zip(layers, inputs, weights):
+        wb = oracle.binarize(w)
+        oracle.conv(x, wb.e, wb.alpha, wb.beta, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad), details=False)
+        ops += L.binary_ops
+    return time.perf_counter() - t0, ops
+
+
+def oracle_sample(batch, dense):
+    import oracle
+    from dab_synth import configs
+    threads = os.cpu_count() or 1
+    oracle.set_threads(threads)
+    layers = configs.config5(batch)
+    inputs = [L.inputs(stream=i, dense=dense) for i, L in enumerate(layers)]
+    weights = [L.weights(stream=i) for i, L in enumerate(layers)]
+    return layers, inputs, weights, threads
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    batch = 2
+    layers, inputs, weights, threads = oracle_sample(batch, args.dense)
+    for _ in range(max(args.warmup, 0)):
+        oracle_pass(layers, inputs, weights)
+    t, ops = 0.0, 0
+    for _ in range(args.steps):
+        dt, o = oracle_pass(layers, inputs, weights)
+        t += dt
+        ops += o
+    value = ops / t / 1e12
+    sample = "all 16 layers of the workload at batch %d (of 256) per step, every patch and filter" % batch
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(args, batch_override=batch),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def select_layers(layers, args):
+    if not args.layers:
+        return layers
+    want = set(args.layers.split(","))
+    sel = [L for L in layers if L.name in want]
+    if not sel:
+        raise SystemExit("no layer named in --layers; names: " + ",".join(L.name for L in layers))
+    return sel
+
+
+def workload_config(args, batch_override=None):
+    b = batch_override if batch_override is not None else args.batch
+    return {"layers": args.layers or "all 16",
+            "workload": "config 5: ResNet-18-shaped stack of 16 binarized 3x3 convolutions (64/128/256/512 channels, "
+                        "56/28/14/7 px), per-filter and per-patch distribution-aware binarization, AND-popcount contraction",
+            "batch_per_gpu": b, "inputs": "dense N(0,1)" if args.dense else "post-ReLU half-normal, 60% exact zeros",
+            "weights": "N(0, 0.02^2)", "l2": "no flush: a step streams >3 GB of distinct inputs and outputs, L2 is 126 MB",
+            "parallelism": "replicas" if args.gpus > 1 else "single GPU"}
+
+
+# ------------------------------------------------------------------------------------------------------------
+# The CUDA path
+# ------------------------------------------------------------------------------------------------------------
+def run_dab(args):
+    import numpy as np
+    import torch
+    import paper_1804_02941_b200 as dab
+    from dab_synth import configs
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    dab.lib()
+    hbm_peak, peak_src, sm_max_mhz = load_peaks()
+
+    layers = select_layers(configs.config5(args.batch), args)
+    # one host tensor per distinct input shape (pinned: it is also the source of the end-to-end copies);
+    # every layer gets its own device copy, shifted along the batch axis so that no two layers share memory
+    host_x = {}
+    for L in layers:
+        if L.x_shape() not in host_x:
+            host_x[L.x_shape()] = torch.from_numpy(L.inputs(stream=100 * rank + len(host_x), dense=args.dense)).pin_memory()
+    stream = torch.cuda.Stream(device=dev)
+    work = []
+    max_patches_words = max(L.patches * dab.dab_default_ld(L.n) for L in layers)
+    max_patches = max(L.patches for L in layers)
+    max_y = max(L.patches * L.Cout for L in layers)
+    pK = torch.empty(max_patches, dtype=torch.int32, device=dev)
+    pg = torch.empty(max_patches, dtype=torch.float32, device=dev)
+    pd = torch.empty(max_patches, dtype=torch.float32, device=dev)
+    pm_flat = torch.empty(max_patches_words, dtype=torch.int32, device=dev)
+    y_flat = torch.empty(max_y, dtype=torch.float32, device=dev)
+    for i, L in enumerate(layers):
+        x = torch.roll(host_x[L.x_shape()].to(dev), shifts=i, dims=0).contiguous()
+        w = torch.from_numpy(L.weights(stream=100 * rank + i)).to(dev)
+        ld = dab.dab_default_ld(L.n)
+        wc = dab.Coded(torch.empty((L.Cout, ld), dtype=torch.int32, device=dev), torch.empty(L.Cout, dtype=torch.int32, device=dev),
+                       torch.empty(L.Cout, dtype=torch.float32, device=dev), torch.empty(L.Cout, dtype=torch.float32, device=dev),
+                       torch.empty(L.Cout, dtype=torch.int32, device=dev), L.n)
+        desc = dab.make_desc(L.x_shape(), L.Cout, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad))
+        pm = pm_flat[: L.patches * ld].view(L.patches, ld)
+        y = y_flat[: L.patches * L.Cout].view(L.N, L.Cout, L.Ho, L.Wo)
+        work.append((L, x, w, wc, desc, pm, y))
+    torch.cuda.synchronize()
+
+    def step(events=None):
+        for li, (L, x, w, wc, desc, pm, y) in enumerate(work):
+            if events is not None:
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                ev[0].record(stream)
+            dab.dab_binarize_into(w, wc.K, wc.alpha, wc.beta, wc.mask, wc.flags, stream=stream)
+            if events is not None:
+                ev[1].record(stream)
+            dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, None, stream=stream)
+            if events is not None:
+                ev[2].record(stream)
+            dab.dab_binary_conv_contract(desc, pm, pK, pg, pd, wc, y, None, stream=stream)
+            if events is not None:
+                ev[3].record(stream)
+                events.append((li, ev))
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    stream.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    events = []
+    barrier()
+    torch.cuda.synchronize()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for _ in range(args.steps):
+        step(events)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    ops_per_step = sum(L.binary_ops for L in layers)
+    value = world * ops_per_step * args.steps / (total_ms * 1e-3) / 1e12
+
+    # per-kernel device time inside the timed region
+    k_ms = {"binarize_rows": 0.0, "binarize_patches": 0.0, "contract": 0.0}
+    for li, ev in events:
+        k_ms["binarize_rows"] += ev[0].elapsed_time(ev[1])
+        k_ms["binarize_patches"] += ev[1].elapsed_time(ev[2])
+        k_ms["contract"] += ev[2].elapsed_time(ev[3])
+    launches_per_kind = args.steps * len(layers)
+
+    # algorithmic bytes of the patch coder: every input element read once (4 B), per patch the packed mask
+    # (4*ceil(n/32) B) and K, gamma, delta (12 B) written
+    patch_bytes = sum(4 * L.N * L.C * L.H * L.W + L.patches * (4 * dab.dab_words_per_row(L.n) + 12) for L in layers)
+    binarize_gbs = patch_bytes * args.steps / (k_ms["binarize_patches"] * 1e-3) / 1e9
+    roofline = {"kernel": "binarize_patches_kernel", "bound": "hbm", "achieved": binarize_gbs, "peak": hbm_peak,
+                "unit": "GB/s", "frac": binarize_gbs / hbm_peak, "traffic": None, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch_avg": patch_bytes / len(layers),
+                "avg_launch_ms": k_ms["binarize_patches"] / launches_per_kind,
+                "share_of_step": k_ms["binarize_patches"] / sum(k_ms.values())}
+
+    # contraction: integer AND/POPC/IADD; peak measured live with independent popcount chains
+    sink = torch.empty(SM_COUNT * 8 * 256, dtype=torch.int32, device=dev)
+    with torch.cuda.stream(stream):
+        dab.dab_popc_probe(SM_COUNT * 8, 2000, sink, stream=stream)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        dab.dab_popc_probe(SM_COUNT * 8, 20000, sink, stream=stream)
+        p1.record(stream)
+    stream.synchronize()
+    probe_words = SM_COUNT * 8 * 256 * 20000 * 16 / (p0.elapsed_time(p1) * 1e-3)
+    contract_tops = ops_per_step * args.steps / (k_ms["contract"] * 1e-3) / 1e12
+    popc_peak_measured = probe_words * 64 / 1e12
+    popc_peak_derived = POPC_PER_CLK_PER_SM * SM_COUNT * sm_max_mhz * 1e6 * 64 / 1e12
+    roofline_contract = {"kernel": "binary_gemm_kernel", "bound": "alu", "achieved": contract_tops,
+                         "peak": popc_peak_derived, "unit": "TOPS-equiv", "frac": contract_tops / popc_peak_derived,
+                         "peak_measured_by_probe": popc_peak_measured,
+                         "peak_source": "16 popc/clk/SM x 148 SMs x %.0f MHz x 64 binary ops per word" % sm_max_mhz,
+                         "avg_launch_ms": k_ms["contract"] / launches_per_kind,
+                         "share_of_step": k_ms["contract"] / sum(k_ms.values())}
+
+    # end to end: host tensors in pinned memory, copies inside the timed region, through the host entry point
+    e2e = None
+    if not args.no_e2e:
+        max_ws = max(dab.dab_binary_conv_host_workspace(desc) for (_, _, _, _, desc, _, _) in work)
+        ws = torch.empty(max_ws, dtype=torch.uint8, device=dev)
+        y_host = torch.empty(max_y, dtype=torch.float32).pin_memory()
+        h2d = sum(4 * L.N * L.C * L.H * L.W for L in layers)
+        d2h = sum(4 * L.patches * L.Cout for L in layers)
+
+        def e2e_step():
+            for (L, x, w, wc, desc, pm, y) in work:
+                dab.dab_binarize_into(w, wc.K, wc.alpha, wc.beta, wc.mask, wc.flags, stream=stream)
+                yh = y_host[: L.patches * L.Cout].view(L.N, L.Cout, L.Ho, L.Wo)
+                dab.dab_binary_conv_host(host_x[L.x_shape()], wc, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad),
+                                         y_host=yh, workspace=ws, stream=stream)
+        e2e_step()
+        barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        e2e = {"value": world * ops_per_step * args.e2e_steps / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * e2e_s / args.e2e_steps}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        b = args.cpu_sample_batch
+        ls, xs, wts, threads = oracle_sample(b, args.dense)
+        dt, ops = oracle_pass(ls, xs, wts)
+        cpu_baseline = {"value": ops / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
+                        "sample": "all 16 layers at batch %d (of %d), every patch and filter, one pass" % (b, args.batch)}
+
+    if rank == 0:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+               "scaling": "weak", "vs_baseline": None, "dtype": "u32 popcount + f64 objective/rescale",
+               "data": "synthetic", "config": workload_config(args), "clocks": clocks, "e2e": e2e,
+               "gpu_launches": 3 * launches_per_kind,
+               "kernel_ms_per_step": {k: v / args.steps for k, v in k_ms.items()},
+               "binarize_gbs": binarize_gbs, "roofline": roofline, "roofline_contraction": roofline_contract,
+               "cpu_baseline": cpu_baseline}
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_dab(args)
+
+
+if __name__ == "__main__":
+    main()

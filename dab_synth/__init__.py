@@ -17,6 +17,9 @@ half-normal with 60 % exact zeros, stroke images are a zero background with
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 DEFAULT_SEED = 180402941
@@ -24,17 +27,19 @@ DEFAULT_SEED = 180402941
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
 _M1 = np.uint64(0xBF58476D1CE4E5B9)
 _M2 = np.uint64(0x94D049BB133111EB)
-_CHUNK = 1 << 22
+_CHUNK = 1 << 18
 
 
 def _mix(z: np.ndarray) -> np.ndarray:
-    """splitmix64 output function (Steele, Lea, Flood 2014), elementwise on uint64."""
-    z = z.copy()
-    z ^= z >> np.uint64(30)
+    """splitmix64 output function (Steele, Lea, Flood 2014), elementwise on uint64, in place."""
+    t = z >> np.uint64(30)
+    z ^= t
     z *= _M1
-    z ^= z >> np.uint64(27)
+    np.right_shift(z, np.uint64(27), out=t)
+    z ^= t
     z *= _M2
-    z ^= z >> np.uint64(31)
+    np.right_shift(z, np.uint64(31), out=t)
+    z ^= t
     return z
 
 
@@ -49,28 +54,50 @@ def raw_u64(seed: int, stream: int, start: int, count: int, lane: int = 0) -> np
     """64 random bits for counters start..start+count-1 of (seed, stream, lane)."""
     key = _stream_key(seed, stream * 8 + lane)
     with np.errstate(over="ignore"):
-        ctr = np.arange(start, start + count, dtype=np.uint64)
-        return _mix(key + (ctr + np.uint64(1)) * _GOLDEN)
+        ctr = np.arange(start + 1, start + count + 1, dtype=np.uint64)
+        ctr *= _GOLDEN
+        ctr += key
+        return _mix(ctr)
 
 
 def uniform01(seed: int, stream: int, start: int, count: int, lane: int = 0) -> np.ndarray:
     """float64 uniform in the open interval (0, 1): (top 53 bits + 0.5) / 2^53."""
-    u = raw_u64(seed, stream, start, count, lane) >> np.uint64(11)
-    return (u.astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
+    u = raw_u64(seed, stream, start, count, lane)
+    u >>= np.uint64(11)
+    f = u.astype(np.float64)
+    f += 0.5
+    f *= 1.0 / 9007199254740992.0
+    return f
 
 
 def _normal_block(seed, stream, start, count):
     u1 = uniform01(seed, stream, start, count, lane=0)
     u2 = uniform01(seed, stream, start, count, lane=1)
-    return np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+    np.log(u1, out=u1)
+    u1 *= -2.0
+    np.sqrt(u1, out=u1)
+    u2 *= 2.0 * np.pi
+    np.cos(u2, out=u2)
+    u1 *= u2
+    return u1
 
 
 def _fill(shape, fn) -> np.ndarray:
+    """Evaluates fn(start, count) over chunks of the flattened array (chunks are independent: any order)."""
     total = int(np.prod(shape, dtype=np.int64)) if len(shape) else 1
     out = np.empty(total, dtype=np.float32)
-    for s in range(0, total, _CHUNK):
+
+    def one(s):
         c = min(_CHUNK, total - s)
         out[s:s + c] = fn(s, c)
+
+    starts = range(0, total, _CHUNK)
+    if len(starts) <= 1:
+        for s in starts:
+            one(s)
+    else:
+        with ThreadPoolExecutor(max_workers=min(len(starts), os.cpu_count() or 1, 16)) as ex:
+            list(ex.map(one, starts))
     return out.reshape(shape)
 
 

@@ -131,6 +131,25 @@ dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const ui
                            void* stream);
 
 /*
+ * The two stages of dab_binary_conv as calls of their own (dab_binary_conv runs exactly these two, in this
+ * order, on the same stream).  A caller that wants the patch codes of an activation tensor once and several
+ * contractions against them, or that times the stages separately, uses these.
+ *
+ * dab_binarize_patches — Section 4.1 / Algorithm 1 applied to every patch of d_x (patch definition, element
+ * order and zero padding as in dab_binary_conv); outputs as the optional outputs of dab_binary_conv, here
+ * required except d_pflags.
+ *
+ * dab_binary_conv_contract — Section 4.3.2: the coded patches against the coded filters, result in NCHW.
+ * d_p11 (patches x Cout int32) may be NULL.
+ */
+dab_status dab_binarize_patches(const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
+                                float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream);
+dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d_pmask, int32_t ldp,
+                                    const int32_t* d_pK, const float* d_pgamma, const float* d_pdelta,
+                                    const uint32_t* d_wmask, int32_t ldw, const int32_t* d_wK, const float* d_walpha,
+                                    const float* d_wbeta, float* d_y, int32_t* d_p11, void* stream);
+
+/*
  * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory: copies h_x
  * to the device, runs dab_binary_conv, copies the result to h_y, all on `stream`, and returns after
  * the stream has drained.  Pinned host memory makes the copies asynchronous to other streams.

@@ -21,7 +21,8 @@ ROW_DEGENERATE = 1
 ROW_NONFINITE = 2
 
 EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_binarize", "dab_pack", "dab_binary_gemm",
-           "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binary_conv_host_workspace",
+           "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
+           "dab_binary_conv_contract", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_popc_probe")
 
 
@@ -59,6 +60,8 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_workspace.argtypes = [vp]
         L.dab_binary_conv_host_workspace.argtypes = [vp]
         L.dab_binary_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp, vp, vp, vp, i32, vp, vp, vp]
+        L.dab_binarize_patches.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp]
+        L.dab_binary_conv_contract.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.dab_binary_conv_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
         _lib = L
@@ -230,6 +233,22 @@ def dab_binary_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), 
                                _ptr(det.p11) if det else None, _stream(stream))
     _check(st, "dab_binary_conv")
     return (y, det) if details else y
+
+
+def dab_binarize_patches(desc: ConvDesc, x: torch.Tensor, pK, pgamma, pdelta, pmask, pflags=None, stream=None) -> None:
+    """Stage 1 of dab_binary_conv with caller-provided outputs (pmask: patches x ld int32)."""
+    st = lib().dab_binarize_patches(C.byref(desc), _ptr(x), _ptr(pK), _ptr(pgamma), _ptr(pdelta), _ptr(pmask),
+                                    pmask.stride(0), _ptr(pflags), _stream(stream))
+    _check(st, "dab_binarize_patches")
+
+
+def dab_binary_conv_contract(desc: ConvDesc, pmask, pK, pgamma, pdelta, w: Coded, y: torch.Tensor, p11=None,
+                             stream=None) -> None:
+    """Stage 2 of dab_binary_conv: coded patches x coded filters -> y (NCHW)."""
+    st = lib().dab_binary_conv_contract(C.byref(desc), _ptr(pmask), pmask.stride(0), _ptr(pK), _ptr(pgamma),
+                                        _ptr(pdelta), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha), _ptr(w.beta),
+                                        _ptr(y), _ptr(p11), _stream(stream))
+    _check(st, "dab_binary_conv_contract")
 
 
 def dab_binary_conv_host(x_host: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0),

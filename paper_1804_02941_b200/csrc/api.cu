@@ -124,43 +124,66 @@ size_t dab_binary_conv_workspace(const dab_conv_desc* desc) {
   return conv_scratch(g).total;
 }
 
+dab_status dab_binarize_patches(const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
+                                float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream) {
+  if (!desc) return DAB_ERR_INVALID_ARG;
+  if (desc->C > 0 && desc->kh > 0 && desc->kw > 0 && (int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N)
+    return DAB_ERR_UNSUPPORTED;
+  ConvGeom g;
+  if (!conv_geom(desc, &g)) return DAB_ERR_INVALID_ARG;
+  if (!d_x || !d_pK || !d_pgamma || !d_pdelta || !d_pmask) return DAB_ERR_INVALID_ARG;
+  if (ldp < dab_words_per_row(g.n) || (ldp & 3) || !aligned16(d_pmask)) return DAB_ERR_INVALID_ARG;
+  return from_cuda(launch_binarize_patches(*desc, g.Ho, g.Wo, d_x, d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags,
+                                           static_cast<cudaStream_t>(stream)));
+}
+
+dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d_pmask, int32_t ldp,
+                                    const int32_t* d_pK, const float* d_pgamma, const float* d_pdelta,
+                                    const uint32_t* d_wmask, int32_t ldw, const int32_t* d_wK, const float* d_walpha,
+                                    const float* d_wbeta, float* d_y, int32_t* d_p11, void* stream) {
+  ConvGeom g;
+  if (!conv_geom(desc, &g)) return DAB_ERR_INVALID_ARG;
+  if (!d_pmask || !d_pK || !d_pgamma || !d_pdelta || !d_wmask || !d_wK || !d_walpha || !d_wbeta || !d_y)
+    return DAB_ERR_INVALID_ARG;
+  int32_t wd = dab_words_per_row(g.n);
+  if (ldp < wd || (ldp & 3) || !aligned16(d_pmask) || ldw < wd || (ldw & 3) || !aligned16(d_wmask))
+    return DAB_ERR_INVALID_ARG;
+  if (desc->Cout > 65535 * 64) return DAB_ERR_UNSUPPORTED;
+  GemmArgs a;
+  a.M = g.patches; a.N = desc->Cout; a.n = g.n; a.words = (wd + 3) / 4 * 4;
+  a.A = d_pmask; a.lda = ldp; a.KA = d_pK; a.gamma = d_pgamma; a.delta = d_pdelta;
+  a.B = d_wmask; a.ldb = ldw; a.KB = d_wK; a.alpha = d_walpha; a.beta = d_wbeta;
+  a.C = d_y;
+  int64_t HoWo = (int64_t)g.Ho * g.Wo;
+  a.map.inner = HoWo; a.map.outer_stride = (int64_t)desc->Cout * HoWo; a.map.row_stride = 1; a.map.col_stride = HoWo;
+  a.p11 = d_p11; a.ldp = desc->Cout;
+  return from_cuda(launch_gemm(a, /*lanes_along_rows=*/true, static_cast<cudaStream_t>(stream)));
+}
+
 dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
                            const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
                            void* d_workspace, size_t workspace_bytes, int32_t* d_pK, float* d_pgamma,
                            float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, int32_t* d_p11,
                            void* stream) {
   if (!desc) return DAB_ERR_INVALID_ARG;
-  if ((int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N && desc->C > 0 && desc->kh > 0 && desc->kw > 0)
+  if (desc->C > 0 && desc->kh > 0 && desc->kw > 0 && (int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N)
     return DAB_ERR_UNSUPPORTED;
   ConvGeom g;
   if (!conv_geom(desc, &g)) return DAB_ERR_INVALID_ARG;
   if (!d_x || !d_wmask || !d_wK || !d_walpha || !d_wbeta || !d_y) return DAB_ERR_INVALID_ARG;
-  if (ldw < dab_words_per_row(g.n) || (ldw & 3) || !aligned16(d_wmask)) return DAB_ERR_INVALID_ARG;
   if (d_pmask && (ldp < dab_words_per_row(g.n) || (ldp & 3) || !aligned16(d_pmask))) return DAB_ERR_INVALID_ARG;
   ConvScratch sc = conv_scratch(g);
   if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign) || workspace_bytes < sc.total)
     return DAB_ERR_WORKSPACE;
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(d_workspace);
   int32_t* pK = d_pK ? d_pK : reinterpret_cast<int32_t*>(ws + sc.off_K);
   float* pg = d_pgamma ? d_pgamma : reinterpret_cast<float*>(ws + sc.off_gamma);
   float* pd = d_pdelta ? d_pdelta : reinterpret_cast<float*>(ws + sc.off_delta);
   uint32_t* pm = d_pmask ? d_pmask : reinterpret_cast<uint32_t*>(ws + sc.off_mask);
   int32_t ldm = d_pmask ? ldp : g.ld;
-
-  if (launch_binarize_patches(*desc, g.Ho, g.Wo, d_x, pK, pg, pd, pm, ldm, d_pflags, st) != cudaSuccess)
-    return DAB_ERR_CUDA;
-
-  GemmArgs a;
-  a.M = g.patches; a.N = desc->Cout; a.n = g.n; a.words = (dab_words_per_row(g.n) + 3) / 4 * 4;
-  a.A = pm; a.lda = ldm; a.KA = pK; a.gamma = pg; a.delta = pd;
-  a.B = d_wmask; a.ldb = ldw; a.KB = d_wK; a.alpha = d_walpha; a.beta = d_wbeta;
-  a.C = d_y;
-  int64_t HoWo = (int64_t)g.Ho * g.Wo;
-  a.map.inner = HoWo; a.map.outer_stride = (int64_t)desc->Cout * HoWo; a.map.row_stride = 1; a.map.col_stride = HoWo;
-  a.p11 = d_p11; a.ldp = desc->Cout;
-  return from_cuda(launch_gemm(a, /*lanes_along_rows=*/true, st));
+  dab_status s = dab_binarize_patches(desc, d_x, pK, pg, pd, pm, ldm, d_pflags, stream);
+  if (s != DAB_OK) return s;
+  return dab_binary_conv_contract(desc, pm, ldm, pK, pg, pd, d_wmask, ldw, d_wK, d_walpha, d_wbeta, d_y, d_p11, stream);
 }
 
 size_t dab_binary_conv_host_workspace(const dab_conv_desc* desc) {

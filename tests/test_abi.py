@@ -52,7 +52,7 @@ def test_host_side_helpers_and_validation(lib):
     assert lib.dab_binary_gemm(1, 1, 64, None, 2, None, None, None, None, 4, None, None, None, None, 1, None, 0, None) == 1
     desc = d.make_desc((2, 64, 56, 56), 64, 3, 3, (1, 1), (1, 1))
     assert d.dab_conv_output_size(desc) == (56, 56)
-    assert d.dab_binary_conv_workspace(desc) >= 2 * 56 * 56 * (20 * 4 + 16)
+    assert d.dab_binary_conv_workspace(desc) >= 2 * 56 * 56 * (20 * 4 + 12)
     assert d.dab_binary_conv_host_workspace(desc) > d.dab_binary_conv_workspace(desc)
     assert d.dab_conv_output_size(d.make_desc((1, 1, 225, 225), 64, 15, 15, (3, 3), (0, 0))) == (71, 71)
     assert d.dab_binary_conv_workspace(d.make_desc((1, 64, 8, 8), 4, 17, 17, (1, 1), (8, 8))) == 0   # n > DAB_MAX_N
