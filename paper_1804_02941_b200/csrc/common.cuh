@@ -10,11 +10,16 @@ namespace dab {
 
 constexpr uint32_t kPadKey = 0xFFFFFFFFu;
 
-// Monotone map fp32 -> uint32: a < b  <=>  key(a) < key(b); -0.0 and +0.0 share one key.
+// Monotone map fp32 -> uint32: a < b  <=>  key(a) < key(b); -0.0 and +0.0 share one key (x + 0.0f turns
+// -0.0 into +0.0 and changes nothing else).
 __device__ __forceinline__ uint32_t order_key(float x) {
-  uint32_t b = __float_as_uint(x);
-  if (b == 0x80000000u) b = 0u;
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  uint32_t b = __float_as_uint(__fadd_rn(x, 0.0f));
+  return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
+}
+
+// Keys of non-finite values: +Inf/NaN(+) map to >= 0xFF800000, -Inf/NaN(-) to <= 0x007FFFFF.
+__device__ __forceinline__ bool key_range_nonfinite(uint32_t kmin, uint32_t kmax) {
+  return kmax >= 0xFF800000u || kmin <= 0x007FFFFFu;
 }
 
 __device__ __forceinline__ float key_value(uint32_t k) {

@@ -1,5 +1,5 @@
-// Core of the row coder: a group of W warps turns one row of n fp32 values (read through an accessor
-// from shared memory) into K, alpha, beta and the packed mask.
+// Core of the row coder: a group of W warps turns one row of n fp32 values (read through an accessor)
+// into K, alpha, beta and the packed mask.
 //
 // Steps, all inside the group:
 //   1. compaction  - keys of the non-zero values go to a scratch array; exact zeros are only counted.
@@ -7,12 +7,15 @@
 //                    as one block of z elements with sum 0 at its place in the sorted order.
 //   2. sort        - bitonic network on registers, E keys per thread, blocked layout (thread t owns
 //                    sorted positions t*E .. t*E+E-1): strides below E stay inside a thread, strides
-//                    below 32E use warp shuffles, larger ones go through shared memory.
+//                    below 32E use warp shuffles, larger ones go through shared memory.  Every merge
+//                    starts with a mirror stage so that all compare-exchanges sort upwards.
 //   3. scan        - fp64 running sums of the sorted values (thread-local, then across the group).
-//   4. objective   - D_s of Algorithm 1 at every split between distinct values, arg-max with
-//                    "largest s wins ties", done on (D, s) with integer reductions on the fp64 bits.
-//   5. outputs     - orientation by |mean|, alpha/beta rounded once to fp32, threshold compare and
-//                    ballot for the mask words.
+//   4. objective   - D_s of Algorithm 1 at every split between distinct values.  A first pass uses
+//                    a table of correctly rounded reciprocals instead of divisions (error < 1e-15
+//                    relative) to find the maximum; a second pass evaluates the exactly rounded
+//                    expression only for splits within 1e-13 of that maximum and takes the arg-max of
+//                    (D, s) with "largest s wins ties".
+//   5. outputs     - orientation by |mean|, alpha/beta rounded once to fp32, threshold key for the mask.
 #pragma once
 
 #include "common.cuh"
@@ -20,6 +23,7 @@
 namespace dab {
 
 constexpr uint32_t kZeroKey = 0x80000000u;  // order_key(0.0f)
+constexpr double kBand = 1.0 - 1e-13;       // splits whose approximate objective is below max*kBand cannot win
 
 __device__ __forceinline__ void group_barrier(int bar_id, int threads) {
   if (threads == 32)
@@ -28,47 +32,77 @@ __device__ __forceinline__ void group_barrier(int bar_id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(threads) : "memory");
 }
 
-// Skewed index into the scratch array: makes both the striped accesses of the compaction and the blocked
-// accesses (stride E words between lanes, E a power of two up to 32) free of bank conflicts.
+// Index skew for scratch arrays read with a stride of E words between lanes (E a power of two up to 32).
 __device__ __forceinline__ int skew(int i) { return i + (i >> 5); }
 
+// Ascending bitonic sort of 32*W*E keys, E per thread, blocked layout.
 template <int W, int E>
 __device__ __forceinline__ void group_sort(uint32_t (&r)[E], int tig, uint32_t* xbuf, int bar_id) {
   constexpr int NTOT = 32 * W * E;
+  constexpr int GT = 32 * W;
   const int ibase = tig * E;
 #pragma unroll
   for (int k = 2; k <= NTOT; k <<= 1) {
+    // mirror stage: element i meets element i ^ (k-1); the lower index keeps the minimum
+    if (k <= E) {
 #pragma unroll
-    for (int st = k >> 1; st >= 1; st >>= 1) {
-      if (st >= 32 * E) {  // partner lives in another warp: exchange through shared memory
-        const bool up = (ibase & k) == 0;
-        const bool lower = (ibase & st) == 0;
-        const int partner = tig ^ (st / E);
+      for (int j = 0; j < E; ++j) {
+        const int p = j ^ (k - 1);
+        if (j < p) {
+          uint32_t lo = min(r[j], r[p]), hi = max(r[j], r[p]);
+          r[j] = lo;
+          r[p] = hi;
+        }
+      }
+    } else {
+      const int tx = k / E - 1;  // partner thread = tig ^ tx, partner register = E-1-j
+      const bool lower = (ibase & (k >> 1)) == 0;
+      if (tx >= 32) {
 #pragma unroll
-        for (int j = 0; j < E; ++j) xbuf[j * (32 * W) + tig] = r[j];
-        group_barrier(bar_id, 32 * W);
+        for (int j = 0; j < E; ++j) xbuf[j * GT + tig] = r[j];
+        group_barrier(bar_id, GT);
 #pragma unroll
         for (int j = 0; j < E; ++j) {
-          uint32_t o = xbuf[j * (32 * W) + partner];
-          r[j] = (lower == up) ? min(r[j], o) : max(r[j], o);
+          uint32_t o = xbuf[(E - 1 - j) * GT + (tig ^ tx)];
+          r[j] = lower ? min(r[j], o) : max(r[j], o);
         }
-        group_barrier(bar_id, 32 * W);
-      } else if (st >= E) {  // partner is another lane of this warp
-        const bool up = (ibase & k) == 0;
+        group_barrier(bar_id, GT);
+      } else {
+        uint32_t o[E];
+#pragma unroll
+        for (int j = 0; j < E; ++j) o[j] = __shfl_xor_sync(0xFFFFFFFFu, r[E - 1 - j], tx);
+#pragma unroll
+        for (int j = 0; j < E; ++j) r[j] = lower ? min(r[j], o[j]) : max(r[j], o[j]);
+      }
+    }
+    // half-cleaners: element i meets i ^ st
+#pragma unroll
+    for (int st = k >> 2; st >= 1; st >>= 1) {
+      if (st >= 32 * E) {
+        const bool lower = (ibase & st) == 0;
+#pragma unroll
+        for (int j = 0; j < E; ++j) xbuf[j * GT + tig] = r[j];
+        group_barrier(bar_id, GT);
+#pragma unroll
+        for (int j = 0; j < E; ++j) {
+          uint32_t o = xbuf[j * GT + (tig ^ (st / E))];
+          r[j] = lower ? min(r[j], o) : max(r[j], o);
+        }
+        group_barrier(bar_id, GT);
+      } else if (st >= E) {
         const bool lower = (ibase & st) == 0;
 #pragma unroll
         for (int j = 0; j < E; ++j) {
           uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, r[j], st / E);
-          r[j] = (lower == up) ? min(r[j], o) : max(r[j], o);
+          r[j] = lower ? min(r[j], o) : max(r[j], o);
         }
-      } else {  // both elements in this thread
+      } else {
 #pragma unroll
         for (int j = 0; j < E; ++j) {
           if ((j & st) == 0) {
             uint32_t lo = min(r[j], r[j | st]), hi = max(r[j], r[j | st]);
-            const bool up = (k < E) ? ((j & k) == 0) : ((ibase & k) == 0);
-            r[j] = up ? lo : hi;
-            r[j | st] = up ? hi : lo;
+            r[j] = lo;
+            r[j | st] = hi;
           }
         }
       }
@@ -80,15 +114,16 @@ struct RowResult {
   int K;
   float alpha, beta;
   uint32_t flags;
-  uint32_t tkey;  // mask bit i = (key_i >= tkey) != low_side
+  uint32_t tkey;  // mask bit i = (key_i >= tkey) != (mode == 1)
   int mode;       // 0: e = [w >= t], 1: e = [w < t], 2: empty mask
 };
 
-struct GroupShared {   // per group, in shared memory
+struct GroupShared {   // per group of more than one warp, in shared memory
   double wsum[16];     // per-warp sums
+  double wmax[16];     // per-warp maxima of the approximate objective
   int wneg[16];        // per-warp counts of negative keys
   uint32_t wfirst[17]; // first key of each warp (index W: pad key)
-  unsigned long long wbestD[16];
+  long long wbestD[16];
   int wbestS[16];
   double wbestP[16];
   uint32_t wbestT[16];
@@ -98,22 +133,64 @@ struct GroupShared {   // per group, in shared memory
   RowResult result;
 };
 
-// Sorted keys in r[] (blocked), m real ones, z zeros elsewhere in the row, n row length.
-template <int W, int E>
-__device__ __forceinline__ void group_select(const uint32_t (&r)[E], int m, int z, int n, int tig, GroupShared* gs,
-                                             int bar_id) {
+// Objective with reciprocals from a table (rcp[s] = correctly rounded 1/s): within 1e-15 relative of the
+// exactly rounded expression, both terms being non-negative.
+__device__ __forceinline__ double objective_fast(double P, double T, int s, int n, const double* rcp) {
+  double Q = T - P;
+  return fma(Q * Q, rcp[n - s], (P * P) * rcp[s]);
+}
+
+__device__ __forceinline__ RowResult finish_row(double bP, int bS, uint32_t bT, double T, int n) {
+  double m_lo = __ddiv_rn(bP, (double)bS);
+  double m_hi = __ddiv_rn(__dsub_rn(T, bP), (double)(n - bS));
+  bool low_side = fabs(m_lo) > fabs(m_hi);  // e marks the partition whose mean is larger in magnitude
+  RowResult res;
+  res.K = low_side ? bS : n - bS;
+  res.alpha = (float)(low_side ? m_lo : m_hi);
+  res.beta = (float)(low_side ? m_hi : m_lo);
+  res.flags = 0u;
+  res.tkey = bT;
+  res.mode = low_side ? 1 : 0;
+  return res;
+}
+
+__device__ __forceinline__ RowResult trivial_row(bool bad, float value) {
+  RowResult res;
+  res.K = 0;
+  float c = bad ? __uint_as_float(0x7FC00000u) : value;
+  res.alpha = c;
+  res.beta = c;
+  res.flags = bad ? DAB_ROW_NONFINITE : DAB_ROW_DEGENERATE;
+  res.tkey = 0u;
+  res.mode = 2;
+  return res;
+}
+
+// Objective evaluation over the sorted keys in r[] (blocked layout: this thread owns sorted non-zero positions
+// q0 .. q0+E-1 of m), z zeros elsewhere in the row, n row length.  The result is valid in thread 0 of the group.
+//
+// kTable (rcp = table of n+1 reciprocals): every admissible split gets the fast objective; the splits within
+// 1e-13 of the maximum are the contenders.  One contender (the usual case) wins outright; several are
+// re-evaluated with the exactly rounded expression and compared as (D, s).  Without the table every split is
+// evaluated exactly.
+template <int W, int E, bool kTable>
+__device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m, int z, int n, int tig,
+                                                  GroupShared* gs, int bar_id, const double* rcp) {
+  constexpr int GT = 32 * W;
+  constexpr bool kKeep = kTable && (E <= 8);  // keep fp64 values and fast objectives of this thread in registers
   const int lane = tig & 31, warp = tig >> 5;
   const int q0 = tig * E;
 
-  // thread-local sum and negative count
+  double v[kKeep ? E : 1];
   double local = 0.0;
   int negc = 0;
 #pragma unroll
   for (int j = 0; j < E; ++j) {
-    if (q0 + j < m) {
-      local = __dadd_rn(local, (double)key_value(r[j]));
-      negc += (r[j] < kZeroKey);
-    }
+    const bool in = q0 + j < m;
+    double vj = in ? (double)key_value(r[j]) : 0.0;
+    if (kKeep) v[kKeep ? j : 0] = vj;
+    local = __dadd_rn(local, vj);
+    negc += in && (r[j] < kZeroKey);
   }
   double incl = local;
 #pragma unroll
@@ -131,7 +208,7 @@ __device__ __forceinline__ void group_select(const uint32_t (&r)[E], int m, int 
       gs->wfirst[warp] = r[0];
       if (warp == 0) gs->wfirst[W] = kPadKey;
     }
-    group_barrier(bar_id, 32 * W);
+    group_barrier(bar_id, GT);
     T = 0.0;
     neg = 0;
 #pragma unroll
@@ -148,33 +225,143 @@ __device__ __forceinline__ void group_select(const uint32_t (&r)[E], int m, int 
   }
   double excl = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
   if (lane == 0) excl = 0.0;
-  double P = __dadd_rn(before, excl);
+  const double P0 = __dadd_rn(before, excl);  // sum of everything sorted before this thread's keys
 
-  // objective at every admissible split owned by this thread
+  // Split "after sorted non-zero q": s = q+1 (q negative) or q+1+z; admissible iff q < m, s < n and the next key
+  // differs (the pad key behind the last real key always differs).  Split "after the zeros": s = neg+z, owned
+  // by the thread that holds q == neg, admissible iff z > 0 and neg < m.
+  const bool owns_zero_split = (z > 0) && (neg < m) && (neg >= q0) && (neg < q0 + E);
+
   double bD = -1.0, bP = 0.0;
   int bS = 0;
   uint32_t bT = 0;
+
+  if (kKeep) {
+    double Dj[kKeep ? E : 1];
+    double lmax = 0.0, Pz = 0.0, P = P0;
 #pragma unroll
-  for (int j = 0; j < E; ++j) {
-    const int q = q0 + j;
-    if (q < m) {
-      const uint32_t kc = r[j];
+    for (int j = 0; j < E; ++j) {
+      const int q = q0 + j;
+      if (q == neg) Pz = P;
+      P = __dadd_rn(P, v[kKeep ? j : 0]);
+      const int s = q + 1 + (q >= neg ? z : 0);
       const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
-      if (q == neg && z > 0) {  // split right after the block of zeros (low side: negatives and zeros)
-        const int s = neg + z;
-        if (s <= n - 1) {
-          double D = objective(P, T, s, n);
-          if (D >= bD) { bD = D; bP = P; bS = s; bT = kc; }
+      const bool ok = (q < m) && (s < n) && (r[j] != kn);
+      double D = ok ? objective_fast(P, T, s, n, rcp) : -1.0;
+      Dj[kKeep ? j : 0] = D;
+      lmax = fmax(lmax, D);
+    }
+    const double Dz = owns_zero_split ? objective_fast(Pz, T, neg + z, n, rcp) : -1.0;
+    lmax = fmax(lmax, Dz);
+    // maximum over the group (lmax >= 0: its bit pattern orders like an integer)
+    long long b = __double_as_longlong(lmax);
+    int hi = (int)(b >> 32);
+    int hmax = __reduce_max_sync(0xFFFFFFFFu, hi);
+    unsigned lo = (hi == hmax) ? (unsigned)b : 0u;
+    unsigned lmx = __reduce_max_sync(0xFFFFFFFFu, lo);
+    double gmax = __longlong_as_double(((long long)hmax << 32) | (long long)lmx);
+    if (W > 1) {
+      if (lane == 0) gs->wmax[warp] = gmax;
+      group_barrier(bar_id, GT);
+#pragma unroll
+      for (int w = 0; w < W; ++w) gmax = fmax(gmax, gs->wmax[w]);
+    }
+    const double thr = gmax * kBand;
+    unsigned cmask = (Dz >= thr) ? (1u << E) : 0u;
+#pragma unroll
+    for (int j = 0; j < E; ++j) cmask |= (Dj[kKeep ? j : 0] >= thr) ? (1u << j) : 0u;
+    int total = __reduce_add_sync(0xFFFFFFFFu, __popc(cmask));
+    if (W > 1) {
+      if (lane == 0) gs->wneg[warp] = total;  // wneg is free again
+      group_barrier(bar_id, GT);
+      total = 0;
+#pragma unroll
+      for (int w = 0; w < W; ++w) total += gs->wneg[w];
+    }
+    const bool several = total > 1;
+    while (cmask) {
+      const int j = __ffs(cmask) - 1;
+      cmask &= cmask - 1;
+      double Pc;
+      int s;
+      uint32_t tk;
+      if (j == E) {
+        Pc = Pz;
+        s = neg + z;
+        tk = kPadKey;
+#pragma unroll
+        for (int i = 0; i < E; ++i)
+          if (q0 + i == neg) tk = r[i];  // first key above the zeros
+      } else {
+        Pc = P0;
+        tk = next_first;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+          if (i <= j) Pc = __dadd_rn(Pc, v[kKeep ? i : 0]);
+          if (i == j + 1) tk = r[i];
+        }
+        const int q = q0 + j;
+        s = q + 1 + (q >= neg ? z : 0);
+        if (q == neg - 1 && z > 0) tk = kZeroKey;  // the zeros are the smallest values of the high side
+      }
+      const double D = several ? objective(Pc, T, s, n) : 1.0;
+      if (D > bD || (D == bD && s > bS)) { bD = D; bP = Pc; bS = s; bT = tk; }
+    }
+  } else {
+    double thr = -1.0;
+    if (kTable) {  // pass 1: maximum of the fast objective
+      double P = P0, lmax = 0.0;
+#pragma unroll
+      for (int j = 0; j < E; ++j) {
+        const int q = q0 + j;
+        if (q < m) {
+          const uint32_t kc = r[j];
+          const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
+          if (q == neg && owns_zero_split) lmax = fmax(lmax, objective_fast(P, T, neg + z, n, rcp));
+          P = __dadd_rn(P, (double)key_value(kc));
+          const int s = q + 1 + (q >= neg ? z : 0);
+          if (s < n && kc != kn) lmax = fmax(lmax, objective_fast(P, T, s, n, rcp));
         }
       }
-      P = __dadd_rn(P, (double)key_value(kc));
-      const int s = (q < neg) ? q + 1 : q + 1 + z;
-      const bool last = (q == m - 1);
-      if (s <= n - 1 && (last || kc != kn)) {
-        double D = objective(P, T, s, n);
-        if (D >= bD) {
-          bD = D; bP = P; bS = s;
-          bT = (q == neg - 1 && z > 0) ? kZeroKey : kn;  // smallest value of the high side
+      long long b = __double_as_longlong(lmax);
+      int hi = (int)(b >> 32);
+      int hmax = __reduce_max_sync(0xFFFFFFFFu, hi);
+      unsigned lo = (hi == hmax) ? (unsigned)b : 0u;
+      unsigned lmx = __reduce_max_sync(0xFFFFFFFFu, lo);
+      double gmax = __longlong_as_double(((long long)hmax << 32) | (long long)lmx);
+      if (W > 1) {
+        if (lane == 0) gs->wmax[warp] = gmax;
+        group_barrier(bar_id, GT);
+#pragma unroll
+        for (int w = 0; w < W; ++w) gmax = fmax(gmax, gs->wmax[w]);
+      }
+      thr = gmax * kBand;
+    }
+    // pass 2: exactly rounded objective (of the contenders only, when the table is in use)
+    double P = P0;
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+      const int q = q0 + j;
+      if (q < m) {
+        const uint32_t kc = r[j];
+        const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
+        if (q == neg && owns_zero_split) {
+          const int s = neg + z;
+          if (!kTable || objective_fast(P, T, s, n, rcp) >= thr) {
+            double D = objective(P, T, s, n);
+            if (D >= bD) { bD = D; bP = P; bS = s; bT = kc; }
+          }
+        }
+        P = __dadd_rn(P, (double)key_value(kc));
+        const int s = q + 1 + (q >= neg ? z : 0);
+        if (s < n && kc != kn) {
+          if (!kTable || objective_fast(P, T, s, n, rcp) >= thr) {
+            double D = objective(P, T, s, n);
+            if (D >= bD) {  // ascending s: ">=" keeps the largest s among equal objectives
+              bD = D; bP = P; bS = s;
+              bT = (q == neg - 1 && z > 0) ? kZeroKey : kn;
+            }
+          }
         }
       }
     }
@@ -185,8 +372,8 @@ __device__ __forceinline__ void group_select(const uint32_t (&r)[E], int m, int 
   int hi = (int)(dbits >> 32);
   int hmax = __reduce_max_sync(0xFFFFFFFFu, hi);
   unsigned lo = (hi == hmax) ? (unsigned)dbits : 0u;
-  unsigned lmax = __reduce_max_sync(0xFFFFFFFFu, lo);
-  bool top = (hi == hmax) && ((unsigned)dbits == lmax);
+  unsigned lmax2 = __reduce_max_sync(0xFFFFFFFFu, lo);
+  bool top = (hi == hmax) && ((unsigned)dbits == lmax2);
   int smax = __reduce_max_sync(0xFFFFFFFFu, top ? bS : -1);
   int src = __ffs(__ballot_sync(0xFFFFFFFFu, top && bS == smax)) - 1;
   bD = __shfl_sync(0xFFFFFFFFu, bD, src);
@@ -195,17 +382,17 @@ __device__ __forceinline__ void group_select(const uint32_t (&r)[E], int m, int 
   bS = smax;
   if (W > 1) {
     if (lane == 0) {
-      gs->wbestD[warp] = (unsigned long long)__double_as_longlong(bD);
+      gs->wbestD[warp] = __double_as_longlong(bD);
       gs->wbestS[warp] = bS;
       gs->wbestP[warp] = bP;
       gs->wbestT[warp] = bT;
     }
-    group_barrier(bar_id, 32 * W);
+    group_barrier(bar_id, GT);
     if (tig == 0) {
-      long long best = (long long)gs->wbestD[0];
+      long long best = gs->wbestD[0];
       int bw = 0;
       for (int w = 1; w < W; ++w) {
-        long long d = (long long)gs->wbestD[w];
+        long long d = gs->wbestD[w];
         if (d > best || (d == best && gs->wbestS[w] > gs->wbestS[bw])) { best = d; bw = w; }
       }
       bS = gs->wbestS[bw];
@@ -213,55 +400,47 @@ __device__ __forceinline__ void group_select(const uint32_t (&r)[E], int m, int 
       bT = gs->wbestT[bw];
     }
   }
-  if (tig == 0) {
-    double m_lo = __ddiv_rn(bP, (double)bS);
-    double m_hi = __ddiv_rn(__dsub_rn(T, bP), (double)(n - bS));
-    bool low_side = fabs(m_lo) > fabs(m_hi);  // e marks the partition whose mean is larger in magnitude
-    RowResult res;
-    res.K = low_side ? bS : n - bS;
-    res.alpha = (float)(low_side ? m_lo : m_hi);
-    res.beta = (float)(low_side ? m_hi : m_lo);
-    res.flags = 0u;
-    res.tkey = bT;
-    res.mode = low_side ? 1 : 0;
-    gs->result = res;
-  }
+  RowResult res;
+  if (tig == 0) res = finish_row(bP, bS, bT, T, n);
+  return res;
 }
 
-template <int W, int E>
+// ---------------------------------------------------------------------------------------------------------
+// Groups of several warps (rows longer than 1024 values)
+// ---------------------------------------------------------------------------------------------------------
+template <int W, int E, bool kTable>
 __device__ __noinline__ void group_sort_select(uint32_t* scratch, int m, int z, int n, int tig, GroupShared* gs,
-                                               int bar_id) {
+                                               int bar_id, const double* rcp) {
+  constexpr int GT = 32 * W;
   uint32_t r[E];
 #pragma unroll
-  for (int j = 0; j < E; ++j) {
-    int idx = tig * E + j;
-    r[j] = idx < m ? scratch[skew(idx)] : kPadKey;
+  for (int j = 0; j < E; ++j) {  // the keys are unsorted: any assignment of keys to positions will do
+    int idx = j * GT + tig;
+    r[j] = idx < m ? scratch[idx] : kPadKey;
   }
-  if (W > 1) group_barrier(bar_id, 32 * W);  // scratch is reused for the cross-warp exchanges
+  group_barrier(bar_id, GT);  // scratch is reused for the cross-warp exchanges
   group_sort<W, E>(r, tig, scratch, bar_id);
-  group_select<W, E>(r, m, z, n, tig, gs, bar_id);
+  RowResult res = group_select<W, E, kTable>(r, m, z, n, tig, gs, bar_id, rcp);
+  if (tig == 0) gs->result = res;
 }
 
-// Codes one row.  `value(i)` returns element i (0 <= i < n) from shared memory.  On return gs->result is valid
-// for every thread of the group (after the trailing barrier).
-template <int W, typename Value>
+// Codes one row with a group of W > 1 warps.  `value(i)` returns element i (0 <= i < n).  On return
+// gs->result is valid for every thread of the group.
+template <int W, bool kTable, typename Value>
 __device__ __forceinline__ void group_code_row(Value value, int n, int tig, uint32_t* scratch, GroupShared* gs,
-                                               int bar_id) {
+                                               int bar_id, const double* rcp) {
+  static_assert(W > 1, "single warps use warp_code_row");
   const int lane = tig & 31;
   constexpr int GT = 32 * W;
-  if (W > 1) {
-    if (tig == 0) {
-      gs->count = 0;
-      gs->bad = 0;
-      gs->varied = 0;
-    }
-    group_barrier(bar_id, GT);
+  if (tig == 0) {
+    gs->count = 0;
+    gs->bad = 0;
+    gs->varied = 0;
   }
+  group_barrier(bar_id, GT);
 
-  // 1. compaction of the non-zero keys (order within the scratch array is irrelevant)
+  // compaction of the non-zero keys (their order in the scratch array is irrelevant)
   int bad = 0;
-  int cnt = 0;             // W == 1: the warp's running count lives in a register
-  uint32_t first_key = 0;  // any key of the row, to recognise constant rows
   for (int i0 = (tig >> 5) * 32; i0 < n; i0 += GT) {
     int i = i0 + lane;
     bool nz = false;
@@ -274,65 +453,131 @@ __device__ __forceinline__ void group_code_row(Value value, int n, int tig, uint
     }
     unsigned bal = __ballot_sync(0xFFFFFFFFu, nz);
     if (bal) {
-      int base = cnt;
-      if (W > 1) {
-        if (lane == 0) base = atomicAdd(&gs->count, __popc(bal));
-        base = __shfl_sync(0xFFFFFFFFu, base, 0);
-      } else {
-        cnt += __popc(bal);
-      }
-      if (nz) scratch[skew(base + __popc(bal & ((1u << lane) - 1u)))] = key;
+      int base = 0;
+      if (lane == 0) base = atomicAdd(&gs->count, __popc(bal));
+      base = __shfl_sync(0xFFFFFFFFu, base, 0);
+      if (nz) scratch[base + __popc(bal & ((1u << lane) - 1u))] = key;
     }
   }
-  bad = __any_sync(0xFFFFFFFFu, bad);
-  int m = cnt;
-  if (W > 1) {
-    if (bad && lane == 0) gs->bad = 1;
-    group_barrier(bar_id, GT);
-    m = gs->count;
-    bad = gs->bad;
-  } else {
-    __syncwarp();
-  }
+  if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) gs->bad = 1;
+  group_barrier(bar_id, GT);
+  const int m = gs->count;
   const int z = n - m;
+  bad = gs->bad;
 
-  // constant row: no non-zero at all, or no zero and all keys equal (checked after the sort would be
-  // wasteful: compare every key with the first one instead)
+  // constant row: no non-zero at all, or no zero and all keys equal
   bool constant = (m == 0);
+  uint32_t first_key = 0;
   if (!bad && !constant && z == 0) {
-    first_key = scratch[skew(0)];
+    first_key = scratch[0];
     int diff = 0;
-    for (int i = tig; i < m; i += GT) diff |= (scratch[skew(i)] != first_key);
-    diff = __any_sync(0xFFFFFFFFu, diff);
-    if (W > 1) {
-      if (diff && lane == 0) gs->varied = 1;
-      group_barrier(bar_id, GT);
-      constant = (gs->varied == 0);
-    } else {
-      constant = !diff;
-    }
+    for (int i = tig; i < m; i += GT) diff |= (scratch[i] != first_key);
+    if (__any_sync(0xFFFFFFFFu, diff) && lane == 0) gs->varied = 1;
+    group_barrier(bar_id, GT);
+    constant = (gs->varied == 0);
   }
 
   if (bad || constant) {
-    if (tig == 0) {
-      RowResult res;
-      res.K = 0;
-      float c = bad ? __uint_as_float(0x7FC00000u) : (m == 0 ? 0.0f : key_value(first_key));
-      res.alpha = c;
-      res.beta = c;
-      res.flags = bad ? DAB_ROW_NONFINITE : DAB_ROW_DEGENERATE;
-      res.tkey = 0u;
-      res.mode = 2;
-      gs->result = res;
-    }
+    if (tig == 0) gs->result = trivial_row(bad, m == 0 ? 0.0f : key_value(first_key));
   } else {
     const int per = (m + GT - 1) / GT;  // keys per thread needed
-    if (per <= 4) group_sort_select<W, 4>(scratch, m, z, n, tig, gs, bar_id);
-    else if (per <= 8) group_sort_select<W, 8>(scratch, m, z, n, tig, gs, bar_id);
-    else if (per <= 16) group_sort_select<W, 16>(scratch, m, z, n, tig, gs, bar_id);
-    else group_sort_select<W, 32>(scratch, m, z, n, tig, gs, bar_id);
+    if (per <= 4) group_sort_select<W, 4, kTable>(scratch, m, z, n, tig, gs, bar_id, rcp);
+    else if (per <= 8) group_sort_select<W, 8, kTable>(scratch, m, z, n, tig, gs, bar_id, rcp);
+    else if (per <= 16) group_sort_select<W, 16, kTable>(scratch, m, z, n, tig, gs, bar_id, rcp);
+    else group_sort_select<W, 32, kTable>(scratch, m, z, n, tig, gs, bar_id, rcp);
   }
   group_barrier(bar_id, GT);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// One warp per row (rows of up to 32*R values).  The row's keys stay in registers (R per lane, element
+// i = 32*k + lane in kreg[k]) so that the mask needs no second read of the values.
+// ---------------------------------------------------------------------------------------------------------
+template <int E>
+__device__ __forceinline__ RowResult warp_sort_select(const uint32_t* scratch, int m, int z, int n, int lane,
+                                                      const double* rcp) {
+  uint32_t r[E];
+#pragma unroll
+  for (int j = 0; j < E; ++j) {
+    int idx = j * 32 + lane;
+    r[j] = idx < m ? scratch[idx] : kPadKey;
+  }
+  group_sort<1, E>(r, lane, nullptr, 0);
+  return group_select<1, E, true>(r, m, z, n, lane, nullptr, 0, rcp);
+}
+
+// Rarely taken sizes (more than 256 non-zero keys) are kept out of line so that the registers of the common
+// sizes set the occupancy.
+template <int E>
+__device__ __noinline__ RowResult warp_sort_select_outlined(const uint32_t* scratch, int m, int z, int n, int lane,
+                                                            const double* rcp) {
+  return warp_sort_select<E>(scratch, m, z, n, lane, rcp);
+}
+
+// Returns the result in every lane.  scratch: 32*R words of shared memory owned by the warp; rcp: n+1 reciprocals.
+// kFull: n == 32*R exactly (no bounds tests in the load loop).
+template <int R, bool kFull, typename Value>
+__device__ __forceinline__ RowResult warp_code_row(Value value, int n, int lane, uint32_t* scratch,
+                                                   const double* rcp, uint32_t (&kreg)[R]) {
+  const unsigned lt = (1u << lane) - 1u;
+  uint32_t kmin = kPadKey, kmax = 0u;
+  int m = 0;
+#pragma unroll
+  for (int k = 0; k < R; ++k) {
+    uint32_t key = kZeroKey;
+    if (kFull || k * 32 < n) {
+      const int i = k * 32 + lane;
+      if (kFull || i < n) {
+        key = order_key(value(i));
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
+      }
+      const bool nz = key != kZeroKey;
+      const unsigned bal = __ballot_sync(0xFFFFFFFFu, nz);
+      if (nz) scratch[m + __popc(bal & lt)] = key;  // the non-zero keys, in any order
+      m += __popc(bal);
+    }
+    kreg[k] = key;
+  }
+  kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+  kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+  const bool bad = key_range_nonfinite(kmin, kmax);
+  const int z = n - m;
+  __syncwarp();
+
+  RowResult res;
+  if (bad || kmin == kmax) {
+    res = trivial_row(bad, key_value(kmin));
+  } else {
+    const int per = (m + 31) >> 5;
+    if (per <= 4) res = warp_sort_select<4>(scratch, m, z, n, lane, rcp);
+    else if (per <= 8) res = warp_sort_select<8>(scratch, m, z, n, lane, rcp);
+    else if (R <= 16 || per <= 16) res = warp_sort_select_outlined<16>(scratch, m, z, n, lane, rcp);
+    else res = warp_sort_select_outlined<32>(scratch, m, z, n, lane, rcp);
+    res.K = __shfl_sync(0xFFFFFFFFu, res.K, 0);
+    res.alpha = __shfl_sync(0xFFFFFFFFu, res.alpha, 0);
+    res.beta = __shfl_sync(0xFFFFFFFFu, res.beta, 0);
+    res.flags = 0u;
+    res.tkey = __shfl_sync(0xFFFFFFFFu, res.tkey, 0);
+    res.mode = __shfl_sync(0xFFFFFFFFu, res.mode, 0);
+  }
+  __syncwarp();  // the scratch array may be overwritten by the next row
+  return res;
+}
+
+// Mask words of the row from the keys in registers: word k in lane k (k < R), 0 elsewhere.
+template <int R, bool kFull>
+__device__ __forceinline__ uint32_t warp_mask_words(const uint32_t (&kreg)[R], int n, int lane, const RowResult& res) {
+  uint32_t mine = 0;
+  const bool flip = res.mode == 1;
+#pragma unroll
+  for (int k = 0; k < R; ++k) {
+    // keys beyond n hold the zero key; they are masked here
+    bool bit = (res.mode != 2) && (kFull || k * 32 + lane < n) && ((kreg[k] >= res.tkey) != flip);
+    uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
+    if (lane == k) mine = word;
+  }
+  return mine;
 }
 
 }  // namespace dab
