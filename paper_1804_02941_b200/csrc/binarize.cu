@@ -35,10 +35,6 @@ static int scratch_words_for(int n, int W) {
   return cap;
 }
 
-__device__ __forceinline__ void fill_reciprocals(double* rcp, int n, int tid, int threads) {
-  for (int s = tid; s <= n; s += threads) rcp[s] = s ? __drcp_rn((double)s) : 0.0;
-}
-
 // ---------------------------------------------------------------------------------------------------------
 // Rows of a matrix, one warp per row (n <= 32*R).
 // ---------------------------------------------------------------------------------------------------------
@@ -49,7 +45,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
     uint32_t* __restrict__ flags_out) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
-  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + (n + 2));
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + rcp_table_slots(n));
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t* scratch = scratch_all + warp * (32 * R);
   fill_reciprocals(rcp, n, threadIdx.x, blockDim.x);
@@ -83,7 +79,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
   constexpr int G = WARPS / W;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
-  GroupShared* gs_all = reinterpret_cast<GroupShared*>(rcp + (kTable ? n + 2 : 0));
+  GroupShared* gs_all = reinterpret_cast<GroupShared*>(rcp + (kTable ? rcp_table_slots(n) : 0));
   uint32_t* scratch_all = reinterpret_cast<uint32_t*>(gs_all + G);
 
   const int group = threadIdx.x / (32 * W);
@@ -117,7 +113,7 @@ static cudaError_t launch_rows_warp(const float* values, int64_t rows, int32_t n
                                     float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
                                     cudaStream_t stream) {
   auto kern = binarize_rows_warp_kernel<R, kFull>;
-  size_t smem = sizeof(double) * (n + 2) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
+  size_t smem = sizeof(double) * rcp_table_slots(n) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int64_t blocks = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
@@ -134,7 +130,7 @@ static cudaError_t launch_rows_group(const float* values, int64_t rows, int32_t 
   constexpr int G = WARPS / W;
   auto kern = binarize_rows_group_kernel<W, WARPS, kTable>;
   int sw = scratch_words_for(n, W);
-  size_t smem = (kTable ? sizeof(double) * (n + 2) : 0) + sizeof(GroupShared) * G + sizeof(uint32_t) * (size_t)sw * G;
+  size_t smem = (kTable ? sizeof(double) * rcp_table_slots(n) : 0) + sizeof(GroupShared) * G + sizeof(uint32_t) * (size_t)sw * G;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int64_t blocks = (rows + G - 1) / G;
@@ -233,7 +229,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_patches_warp_ke
   constexpr int THREADS = kWarpsPerCta * 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
-  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + (a.n + 2));
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + rcp_table_slots(a.n));
   float* tile = reinterpret_cast<float*>(scratch_all + kWarpsPerCta * 32 * R);
   const int ch_words = a.in_h * a.pitch;
   uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
@@ -276,7 +272,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
   constexpr int THREADS = WARPS * 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
-  GroupShared* gs_all = reinterpret_cast<GroupShared*>(rcp + (kTable ? a.n + 2 : 0));
+  GroupShared* gs_all = reinterpret_cast<GroupShared*>(rcp + (kTable ? rcp_table_slots(a.n) : 0));
   uint32_t* scratch_all = reinterpret_cast<uint32_t*>(gs_all + G);
   float* tile = reinterpret_cast<float*>(scratch_all + (size_t)G * a.scratch_words);
   const int ch_words = a.in_h * a.pitch;
@@ -355,7 +351,7 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
 
 template <int R, bool kFull>
 static cudaError_t launch_patches_warp(PatchArgs& a, cudaStream_t stream) {
-  size_t fixed = sizeof(double) * (a.n + 2) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
+  size_t fixed = sizeof(double) * rcp_table_slots(a.n) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
   return launch_patches(binarize_patches_warp_kernel<R, kFull>, a, fixed, kWarpsPerCta * 32, stream);
 }
 
@@ -363,7 +359,7 @@ template <int W, int WARPS, bool kTable>
 static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream) {
   constexpr int G = WARPS / W;
   a.scratch_words = scratch_words_for(a.n, W);
-  size_t fixed = (kTable ? sizeof(double) * (a.n + 2) : 0) + sizeof(GroupShared) * G +
+  size_t fixed = (kTable ? sizeof(double) * rcp_table_slots(a.n) : 0) + sizeof(GroupShared) * G +
                  sizeof(uint32_t) * (size_t)a.scratch_words * G;
   return launch_patches(binarize_patches_group_kernel<W, WARPS, kTable>, a, fixed, WARPS * 32, stream);
 }

@@ -133,11 +133,21 @@ struct GroupShared {   // per group of more than one warp, in shared memory
   RowResult result;
 };
 
-// Objective with reciprocals from a table (rcp[s] = correctly rounded 1/s): within 1e-15 relative of the
-// exactly rounded expression, both terms being non-negative.
+// Table of correctly rounded reciprocals 1/s, s = 1..n.  Lanes of a warp look up values of s that are E apart
+// (E = 4, 8, 16, 32), so entry s lives at slot s + s/16: one pad slot per 16 entries spreads such accesses over
+// the banks of shared memory.
+__device__ __forceinline__ int rcp_slot(int s) { return s + (s >> 4); }
+__host__ __device__ inline int rcp_table_slots(int n) { return n + (n >> 4) + 2; }
+
+__device__ __forceinline__ void fill_reciprocals(double* rcp, int n, int tid, int threads) {
+  for (int s = tid; s <= n; s += threads) rcp[rcp_slot(s)] = s ? __drcp_rn((double)s) : 0.0;
+}
+
+// Objective with reciprocals from the table: within 1e-15 relative of the exactly rounded expression, both
+// terms being non-negative.
 __device__ __forceinline__ double objective_fast(double P, double T, int s, int n, const double* rcp) {
   double Q = T - P;
-  return fma(Q * Q, rcp[n - s], (P * P) * rcp[s]);
+  return fma(Q * Q, rcp[rcp_slot(n - s)], (P * P) * rcp[rcp_slot(s)]);
 }
 
 __device__ __forceinline__ RowResult finish_row(double bP, int bS, uint32_t bT, double T, int n) {
@@ -181,15 +191,15 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
   const int lane = tig & 31, warp = tig >> 5;
   const int q0 = tig * E;
 
-  double v[kKeep ? E : 1];
+  double loc[kKeep ? E : 1];  // loc[j] = sum of this thread's sorted values 0..j
   double local = 0.0;
   int negc = 0;
 #pragma unroll
   for (int j = 0; j < E; ++j) {
     const bool in = q0 + j < m;
     double vj = in ? (double)key_value(r[j]) : 0.0;
-    if (kKeep) v[kKeep ? j : 0] = vj;
     local = __dadd_rn(local, vj);
+    if (kKeep) loc[kKeep ? j : 0] = local;
     negc += in && (r[j] < kZeroKey);
   }
   double incl = local;
@@ -235,15 +245,17 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
   double bD = -1.0, bP = 0.0;
   int bS = 0;
   uint32_t bT = 0;
+  bool several = true;
 
   if (kKeep) {
     double Dj[kKeep ? E : 1];
-    double lmax = 0.0, Pz = 0.0, P = P0;
+    // prefix sum up to and including sorted position q0+j: P0 + loc[j] (the same expression wherever it is needed)
+    double lmax = 0.0, Pz = P0;
 #pragma unroll
     for (int j = 0; j < E; ++j) {
       const int q = q0 + j;
-      if (q == neg) Pz = P;
-      P = __dadd_rn(P, v[kKeep ? j : 0]);
+      const double P = __dadd_rn(P0, loc[kKeep ? j : 0]);
+      if (q + 1 == neg) Pz = P;  // sum of the negatives (P0 itself when neg == q0)
       const int s = q + 1 + (q >= neg ? z : 0);
       const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
       const bool ok = (q < m) && (s < n) && (r[j] != kn);
@@ -278,7 +290,7 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
 #pragma unroll
       for (int w = 0; w < W; ++w) total += gs->wneg[w];
     }
-    const bool several = total > 1;
+    several = total > 1;
     while (cmask) {
       const int j = __ffs(cmask) - 1;
       cmask &= cmask - 1;
@@ -293,13 +305,14 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
         for (int i = 0; i < E; ++i)
           if (q0 + i == neg) tk = r[i];  // first key above the zeros
       } else {
-        Pc = P0;
+        double lj = 0.0;
         tk = next_first;
 #pragma unroll
         for (int i = 0; i < E; ++i) {
-          if (i <= j) Pc = __dadd_rn(Pc, v[kKeep ? i : 0]);
+          if (i == j) lj = loc[kKeep ? i : 0];
           if (i == j + 1) tk = r[i];
         }
+        Pc = __dadd_rn(P0, lj);
         const int q = q0 + j;
         s = q + 1 + (q >= neg ? z : 0);
         if (q == neg - 1 && z > 0) tk = kZeroKey;  // the zeros are the smallest values of the high side
@@ -367,19 +380,25 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
     }
   }
 
-  // arg-max of (D, s): D >= 0 (or -1 for "none"), so its bits order like a signed 64-bit integer
-  long long dbits = __double_as_longlong(bD);
-  int hi = (int)(dbits >> 32);
-  int hmax = __reduce_max_sync(0xFFFFFFFFu, hi);
-  unsigned lo = (hi == hmax) ? (unsigned)dbits : 0u;
-  unsigned lmax2 = __reduce_max_sync(0xFFFFFFFFu, lo);
-  bool top = (hi == hmax) && ((unsigned)dbits == lmax2);
-  int smax = __reduce_max_sync(0xFFFFFFFFu, top ? bS : -1);
-  int src = __ffs(__ballot_sync(0xFFFFFFFFu, top && bS == smax)) - 1;
+  int src;
+  if (!several) {  // a single contender in the whole group: no comparison needed
+    const unsigned own = __ballot_sync(0xFFFFFFFFu, bD > 0.0);
+    src = own ? __ffs(own) - 1 : 0;
+  } else {
+    // arg-max of (D, s): D >= 0 (or -1 for "none"), so its bits order like a signed 64-bit integer
+    long long dbits = __double_as_longlong(bD);
+    int hi = (int)(dbits >> 32);
+    int hmax = __reduce_max_sync(0xFFFFFFFFu, hi);
+    unsigned lo = (hi == hmax) ? (unsigned)dbits : 0u;
+    unsigned lmax2 = __reduce_max_sync(0xFFFFFFFFu, lo);
+    bool top = (hi == hmax) && ((unsigned)dbits == lmax2);
+    int smax = __reduce_max_sync(0xFFFFFFFFu, top ? bS : -1);
+    src = __ffs(__ballot_sync(0xFFFFFFFFu, top && bS == smax)) - 1;
+  }
   bD = __shfl_sync(0xFFFFFFFFu, bD, src);
   bP = __shfl_sync(0xFFFFFFFFu, bP, src);
   bT = __shfl_sync(0xFFFFFFFFu, bT, src);
-  bS = smax;
+  bS = __shfl_sync(0xFFFFFFFFu, bS, src);
   if (W > 1) {
     if (lane == 0) {
       gs->wbestD[warp] = __double_as_longlong(bD);
