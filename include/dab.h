@@ -161,6 +161,31 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
                                 void* d_workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * dab_binary_conv_static — dab_binary_conv without a workspace argument.  The paper has no counterpart: this
+ * entry point exists for callers that cannot allocate device memory themselves, for example code running
+ * inside a plugin or callback interface that hands it device pointers for inputs and outputs only, or a
+ * process whose memory pool is owned by another component and may not be grown after start-up.
+ *
+ * The scratch for the patch codes is a fixed array of DAB_STATIC_SCRATCH_BYTES in device global memory that
+ * belongs to the library image: every GPU on which the library is used holds it until the process exits.
+ * The call allocates and frees nothing.  A layer fits when dab_binary_conv_workspace(desc) is at most
+ * dab_binary_conv_static_capacity(); larger layers are refused with DAB_ERR_UNSUPPORTED (use dab_binary_conv
+ * with your own workspace, or split the batch).  Inputs, outputs and their meaning are those of
+ * dab_binary_conv; the optional outputs are not available here.
+ *
+ * The first call on each device looks up the device address of the array (a synchronous runtime query made
+ * with that device current); make that first call outside any stream capture.  All calls on a device share
+ * the one array and it keeps whatever the last call left in it: nothing in it needs clearing because each call
+ * overwrites all it reads, but two calls whose kernels can overlap on the GPU (different streams, no ordering
+ * between them) race on it and must be serialised by the caller.
+ */
+#define DAB_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+size_t dab_binary_conv_static_capacity(void);
+dab_status dab_binary_conv_static(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                                  const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
+                                  void* stream);
+
+/*
  * dab_popc_probe — measurement aid, not part of the method: runs `iters` rounds of independent
  * AND + population-count + add chains in every thread of a grid of `blocks` x 256 threads and
  * writes one word per thread to d_sink (blocks*256 words), so that a caller timing it obtains the

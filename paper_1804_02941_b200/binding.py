@@ -23,7 +23,7 @@ ROW_NONFINITE = 2
 EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_binarize", "dab_pack", "dab_binary_gemm",
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_binary_conv_host_workspace",
-           "dab_binary_conv_host", "dab_popc_probe")
+           "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe")
 
 
 class DabError(RuntimeError):
@@ -63,6 +63,9 @@ def lib() -> C.CDLL:
         L.dab_binarize_patches.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp]
         L.dab_binary_conv_contract.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.dab_binary_conv_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.dab_binary_conv_static_capacity.restype = C.c_size_t
+        L.dab_binary_conv_static_capacity.argtypes = []
+        L.dab_binary_conv_static.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
         _lib = L
     return _lib
@@ -269,6 +272,29 @@ def dab_binary_conv_host(x_host: torch.Tensor, w: Coded, kh: int, kw: int, strid
                                     workspace.numel(), _stream(stream))
     _check(st, "dab_binary_conv_host")
     return y_host
+
+
+def dab_binary_conv_static_capacity() -> int:
+    return int(lib().dab_binary_conv_static_capacity())
+
+
+def dab_binary_conv_static(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
+                           y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """dab_binary_conv on the library's built-in scratch array (no workspace; see include/dab.h for its limits).
+
+    Only the output tensor is created here when the caller passes none; the library call itself allocates nothing."""
+    _dev(x, torch.float32, "x")
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous NCHW")
+    Cout = w.mask.shape[0]
+    desc = make_desc(tuple(x.shape), Cout, kh, kw, stride, pad)
+    Ho, Wo = dab_conv_output_size(desc)
+    if y is None:
+        y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=x.device)
+    st = lib().dab_binary_conv_static(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha),
+                                      _ptr(w.beta), _ptr(y), _stream(stream))
+    _check(st, "dab_binary_conv_static")
+    return y
 
 
 def dab_popc_probe(blocks: int, iters: int, sink: torch.Tensor | None = None, stream=None) -> torch.Tensor:
