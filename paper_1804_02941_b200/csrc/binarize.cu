@@ -7,27 +7,6 @@ namespace dab {
 
 constexpr int kWarpsPerCta = 8;
 
-// Writes the packed mask of one row from a group of W > 1 warps: the warps take 32-word batches; lane t keeps
-// word t of a batch so that a batch is stored with one coalesced write.  Words beyond ceil(n/32) are 0.
-template <int W, typename Value>
-__device__ __forceinline__ void group_write_mask(Value value, int n, int ld, const RowResult& res, int tig,
-                                                 uint32_t* __restrict__ out) {
-  const int lane = tig & 31, warp = tig >> 5;
-  const bool flip = res.mode == 1;
-  for (int w0 = warp * 32; w0 < ld; w0 += 32 * W) {
-    uint32_t mine = 0;
-    const int wend = min(32, ld - w0);
-    for (int t = 0; t < wend; ++t) {
-      int i = (w0 + t) * 32 + lane;
-      bool bit = false;
-      if (res.mode != 2 && i < n) bit = (order_key(value(i)) >= res.tkey) != flip;
-      uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
-      if (lane == t) mine = word;
-    }
-    if (lane < wend) out[w0 + lane] = mine;
-  }
-}
-
 // Scratch words a group of W warps needs for rows of up to n values (the largest sort capacity reachable).
 static int scratch_words_for(int n, int W) {
   int cap = 128 * W;
@@ -71,7 +50,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
 // ---------------------------------------------------------------------------------------------------------
 // Rows of a matrix, a group of W > 1 warps per row.
 // ---------------------------------------------------------------------------------------------------------
-template <int W, int WARPS, bool kTable>
+template <int W, int WARPS, int R, bool kFull, bool kTable>
 __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
     const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
     float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
@@ -95,7 +74,8 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
   for (int64_t row = (int64_t)blockIdx.x * G + group; row < rows; row += (int64_t)gridDim.x * G) {
     const float* v = values + row * ld_values;
     auto value = [v](int i) { return __ldg(v + i); };
-    group_code_row<W, kTable>(value, n, tig, scratch, gs, bar_id, rcp);
+    uint32_t kreg[R];
+    group_code_row<W, R, kFull, kTable>(value, n, tig, scratch, gs, bar_id, rcp, kreg);
     const RowResult res = gs->result;
     if (tig == 0) {
       K_out[row] = res.K;
@@ -103,7 +83,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
       beta_out[row] = res.beta;
       if (flags_out) flags_out[row] = res.flags;
     }
-    group_write_mask<W>(value, n, ld_mask, res, tig, mask_out + row * (int64_t)ld_mask);
+    group_store_mask<W, R, kFull>(kreg, n, ld_mask, tig, res, mask_out + row * (int64_t)ld_mask);
     group_barrier(bar_id, 32 * W);  // gs->result is overwritten by the next row
   }
 }
@@ -123,12 +103,12 @@ static cudaError_t launch_rows_warp(const float* values, int64_t rows, int32_t n
   return cudaGetLastError();
 }
 
-template <int W, int WARPS, bool kTable>
+template <int W, int WARPS, int R, bool kFull, bool kTable>
 static cudaError_t launch_rows_group(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                      float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
                                      cudaStream_t stream) {
   constexpr int G = WARPS / W;
-  auto kern = binarize_rows_group_kernel<W, WARPS, kTable>;
+  auto kern = binarize_rows_group_kernel<W, WARPS, R, kFull, kTable>;
   int sw = scratch_words_for(n, W);
   size_t smem = (kTable ? sizeof(double) * rcp_table_slots(n) : 0) + sizeof(GroupShared) * G + sizeof(uint32_t) * (size_t)sw * G;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -150,10 +130,15 @@ cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_
   if (n <= 576) return launch_rows_warp<18, false>(DAB_ARGS);
   if (n == 1024) return launch_rows_warp<32, true>(DAB_ARGS);
   if (n <= 1024) return launch_rows_warp<32, false>(DAB_ARGS);
-  if (n <= 2048) return launch_rows_group<2, 8, true>(DAB_ARGS);
-  if (n <= 4096) return launch_rows_group<4, 8, true>(DAB_ARGS);
-  if (n <= 8192) return launch_rows_group<8, 8, true>(DAB_ARGS);
-  return launch_rows_group<16, 16, false>(DAB_ARGS);
+  // rows of exactly 576 values per warp (1152, 2304, 4608, 9216) get the variant without bounds tests
+  if (n == 1152) return launch_rows_group<2, 8, 18, true, true>(DAB_ARGS);
+  if (n <= 2048) return launch_rows_group<2, 8, 32, false, true>(DAB_ARGS);
+  if (n == 2304) return launch_rows_group<4, 8, 18, true, true>(DAB_ARGS);
+  if (n <= 4096) return launch_rows_group<4, 8, 32, false, true>(DAB_ARGS);
+  if (n == 4608) return launch_rows_group<8, 8, 18, true, true>(DAB_ARGS);
+  if (n <= 8192) return launch_rows_group<8, 8, 32, false, true>(DAB_ARGS);
+  if (n == 9216) return launch_rows_group<16, 16, 18, true, false>(DAB_ARGS);
+  return launch_rows_group<16, 16, 32, false, false>(DAB_ARGS);
 #undef DAB_ARGS
 }
 
@@ -266,7 +251,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_patches_warp_ke
   }
 }
 
-template <int W, int WARPS, bool kTable>
+template <int W, int WARPS, int R, bool kFull, bool kTable>
 __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(const PatchArgs a) {
   constexpr int G = WARPS / W;
   constexpr int THREADS = WARPS * 32;
@@ -297,7 +282,8 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
       const int lh = p / t.tw, lw = p % t.tw;
       const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
       auto value = [origin, off](int i) { return origin[off[i]]; };
-      group_code_row<W, kTable>(value, a.n, tig, scratch, gs, bar_id, rcp);
+      uint32_t kreg[R];
+      group_code_row<W, R, kFull, kTable>(value, a.n, tig, scratch, gs, bar_id, rcp, kreg);
       const RowResult res = gs->result;
       const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
       if (tig == 0) {
@@ -306,7 +292,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
         a.pdelta[pi] = res.beta;
         if (a.pflags) a.pflags[pi] = res.flags;
       }
-      group_write_mask<W>(value, a.n, a.ldp, res, tig, a.pmask + pi * (int64_t)a.ldp);
+      group_store_mask<W, R, kFull>(kreg, a.n, a.ldp, tig, res, a.pmask + pi * (int64_t)a.ldp);
       group_barrier(bar_id, 32 * W);
     }
   }
@@ -355,13 +341,13 @@ static cudaError_t launch_patches_warp(PatchArgs& a, cudaStream_t stream) {
   return launch_patches(binarize_patches_warp_kernel<R, kFull>, a, fixed, kWarpsPerCta * 32, stream);
 }
 
-template <int W, int WARPS, bool kTable>
+template <int W, int WARPS, int R, bool kFull, bool kTable>
 static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream) {
   constexpr int G = WARPS / W;
   a.scratch_words = scratch_words_for(a.n, W);
   size_t fixed = (kTable ? sizeof(double) * rcp_table_slots(a.n) : 0) + sizeof(GroupShared) * G +
                  sizeof(uint32_t) * (size_t)a.scratch_words * G;
-  return launch_patches(binarize_patches_group_kernel<W, WARPS, kTable>, a, fixed, WARPS * 32, stream);
+  return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, stream);
 }
 
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
@@ -377,10 +363,14 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   if (a.n <= 576) return launch_patches_warp<18, false>(a, stream);
   if (a.n == 1024) return launch_patches_warp<32, true>(a, stream);
   if (a.n <= 1024) return launch_patches_warp<32, false>(a, stream);
-  if (a.n <= 2048) return launch_patches_group<2, 8, true>(a, stream);
-  if (a.n <= 4096) return launch_patches_group<4, 8, true>(a, stream);
-  if (a.n <= 8192) return launch_patches_group<8, 8, true>(a, stream);
-  return launch_patches_group<16, 16, false>(a, stream);
+  if (a.n == 1152) return launch_patches_group<2, 8, 18, true, true>(a, stream);
+  if (a.n <= 2048) return launch_patches_group<2, 8, 32, false, true>(a, stream);
+  if (a.n == 2304) return launch_patches_group<4, 8, 18, true, true>(a, stream);
+  if (a.n <= 4096) return launch_patches_group<4, 8, 32, false, true>(a, stream);
+  if (a.n == 4608) return launch_patches_group<8, 8, 18, true, true>(a, stream);
+  if (a.n <= 8192) return launch_patches_group<8, 8, 32, false, true>(a, stream);
+  if (a.n == 9216) return launch_patches_group<16, 16, 18, true, false>(a, stream);
+  return launch_patches_group<16, 16, 32, false, false>(a, stream);
 }
 
 }  // namespace dab

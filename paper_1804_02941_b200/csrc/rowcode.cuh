@@ -127,9 +127,9 @@ struct GroupShared {   // per group of more than one warp, in shared memory
   int wbestS[16];
   double wbestP[16];
   uint32_t wbestT[16];
-  int count;           // compaction counter
-  int bad;             // non-finite seen
-  int varied;          // two different keys seen
+  int wcnt[16];        // per-warp counts of non-zero keys
+  uint32_t wkmin[16];  // per-warp smallest and largest key
+  uint32_t wkmax[16];
   RowResult result;
 };
 
@@ -443,61 +443,64 @@ __device__ __noinline__ void group_sort_select(uint32_t* scratch, int m, int z, 
   if (tig == 0) gs->result = res;
 }
 
-// Codes one row with a group of W > 1 warps.  `value(i)` returns element i (0 <= i < n).  On return
-// gs->result is valid for every thread of the group.
-template <int W, bool kTable, typename Value>
+// Codes one row with a group of W > 1 warps.  `value(i)` returns element i (0 <= i < n).  Warp w of the group
+// owns rounds w*R .. w*R+R-1 of the row (element (round)*32 + lane) and keeps their keys in kreg[], so that the
+// mask needs no second read of the values.  kFull: n == 32*W*R exactly.  On return gs->result is valid for
+// every thread of the group.
+template <int W, int R, bool kFull, bool kTable, typename Value>
 __device__ __forceinline__ void group_code_row(Value value, int n, int tig, uint32_t* scratch, GroupShared* gs,
-                                               int bar_id, const double* rcp) {
+                                               int bar_id, const double* rcp, uint32_t (&kreg)[R]) {
   static_assert(W > 1, "single warps use warp_code_row");
-  const int lane = tig & 31;
   constexpr int GT = 32 * W;
-  if (tig == 0) {
-    gs->count = 0;
-    gs->bad = 0;
-    gs->varied = 0;
-  }
-  group_barrier(bar_id, GT);
+  const int lane = tig & 31, warp = tig >> 5;
+  const unsigned lt = (1u << lane) - 1u;
+  const int first = warp * R * 32 + lane;
 
-  // compaction of the non-zero keys (their order in the scratch array is irrelevant)
-  int bad = 0;
-  for (int i0 = (tig >> 5) * 32; i0 < n; i0 += GT) {
-    int i = i0 + lane;
-    bool nz = false;
+  uint32_t kmin = kPadKey, kmax = 0u;
+  int cnt = 0;
+#pragma unroll
+  for (int k = 0; k < R; ++k) {
     uint32_t key = kZeroKey;
-    if (i < n) {
-      float x = value(i);
-      bad |= is_nonfinite(x);
-      key = order_key(x);
-      nz = key != kZeroKey;
+    const int i = first + k * 32;
+    if (kFull || i < n) {
+      key = order_key(value(i));
+      kmin = min(kmin, key);
+      kmax = max(kmax, key);
     }
-    unsigned bal = __ballot_sync(0xFFFFFFFFu, nz);
-    if (bal) {
-      int base = 0;
-      if (lane == 0) base = atomicAdd(&gs->count, __popc(bal));
-      base = __shfl_sync(0xFFFFFFFFu, base, 0);
-      if (nz) scratch[base + __popc(bal & ((1u << lane) - 1u))] = key;
-    }
+    kreg[k] = key;
+    cnt += __popc(__ballot_sync(0xFFFFFFFFu, key != kZeroKey));
   }
-  if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) gs->bad = 1;
+  kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+  kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+  if (lane == 0) {
+    gs->wcnt[warp] = cnt;
+    gs->wkmin[warp] = kmin;
+    gs->wkmax[warp] = kmax;
+  }
   group_barrier(bar_id, GT);
-  const int m = gs->count;
-  const int z = n - m;
-  bad = gs->bad;
-
-  // constant row: no non-zero at all, or no zero and all keys equal
-  bool constant = (m == 0);
-  uint32_t first_key = 0;
-  if (!bad && !constant && z == 0) {
-    first_key = scratch[0];
-    int diff = 0;
-    for (int i = tig; i < m; i += GT) diff |= (scratch[i] != first_key);
-    if (__any_sync(0xFFFFFFFFu, diff) && lane == 0) gs->varied = 1;
-    group_barrier(bar_id, GT);
-    constant = (gs->varied == 0);
+  int base = 0, m = 0;
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    const int c = gs->wcnt[w];
+    if (w < warp) base += c;
+    m += c;
+    kmin = min(kmin, gs->wkmin[w]);
+    kmax = max(kmax, gs->wkmax[w]);
   }
+  // the non-zero keys of all warps, packed (their order is irrelevant)
+#pragma unroll
+  for (int k = 0; k < R; ++k) {
+    const bool nz = kreg[k] != kZeroKey;
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, nz);
+    if (nz) scratch[base + __popc(bal & lt)] = kreg[k];
+    base += __popc(bal);
+  }
+  group_barrier(bar_id, GT);
+  const bool bad = key_range_nonfinite(kmin, kmax);
+  const int z = n - m;
 
-  if (bad || constant) {
-    if (tig == 0) gs->result = trivial_row(bad, m == 0 ? 0.0f : key_value(first_key));
+  if (bad || kmin == kmax) {
+    if (tig == 0) gs->result = trivial_row(bad, key_value(kmin));
   } else {
     const int per = (m + GT - 1) / GT;  // keys per thread needed
     if (per <= 4) group_sort_select<W, 4, kTable>(scratch, m, z, n, tig, gs, bar_id, rcp);
@@ -506,6 +509,26 @@ __device__ __forceinline__ void group_code_row(Value value, int n, int tig, uint
     else group_sort_select<W, 32, kTable>(scratch, m, z, n, tig, gs, bar_id, rcp);
   }
   group_barrier(bar_id, GT);
+}
+
+// Mask words of a row coded by a group: warp w produces words w*R .. w*R+R-1 (word w*R+k in lane k) and stores
+// them with one coalesced write; words from W*R up to ld are written as 0.
+template <int W, int R, bool kFull>
+__device__ __forceinline__ void group_store_mask(const uint32_t (&kreg)[R], int n, int ld, int tig,
+                                                 const RowResult& res, uint32_t* __restrict__ out) {
+  const int lane = tig & 31, warp = tig >> 5;
+  const bool flip = res.mode == 1;
+  uint32_t mine = 0;
+#pragma unroll
+  for (int k = 0; k < R; ++k) {
+    const int i = (warp * R + k) * 32 + lane;
+    bool bit = (res.mode != 2) && (kFull || i < n) && ((kreg[k] >= res.tkey) != flip);
+    uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
+    if (lane == k) mine = word;
+  }
+  const int w = warp * R + lane;
+  if (lane < R && w < ld) out[w] = mine;
+  for (int p = W * R + tig; p < ld; p += 32 * W) out[p] = 0u;
 }
 
 // ---------------------------------------------------------------------------------------------------------
