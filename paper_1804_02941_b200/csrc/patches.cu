@@ -1,0 +1,245 @@
+// The patch coder of dab_binary_conv: the row coder of rowcode.cuh applied to every patch of an NCHW tensor
+// (one warp per patch for up to 1024 values, a group of 2..16 warps beyond).
+#include "rowcode.cuh"
+
+namespace dab {
+
+// ---------------------------------------------------------------------------------------------------------
+// Patches of an NCHW tensor.  A CTA stages the input region under a tile of TH x TW output positions (all
+// channels, zero padding filled in) in shared memory, then codes the tile's patches.
+// Element i of a patch, i = (c*kh + r)*kw + s, sits at tile offset off[i] + patch origin.
+// ---------------------------------------------------------------------------------------------------------
+struct PatchArgs {
+  dab_conv_desc d;
+  int32_t Ho, Wo, n;
+  int32_t TH, TW;          // output positions per tile
+  int32_t in_h, in_w;      // staged rows/columns per channel: (TH-1)*stride_h + kh, (TW-1)*stride_w + kw
+  int32_t pitch;           // words per staged row (>= in_w)
+  int32_t tiles_h, tiles_w;
+  int32_t scratch_words;
+  uint32_t magic_per_ch, magic_in_w;  // ceil(2^32 / d) for d = in_h*in_w and in_w: floor(i/d) = umulhi(i, magic); 0 if d == 1
+  const float* x;
+  int32_t* pK;
+  float* pgamma;
+  float* pdelta;
+  uint32_t* pflags;        // may be null
+  uint32_t* pmask;
+  int32_t ldp;
+};
+
+__device__ __forceinline__ void fill_offsets(const PatchArgs& a, uint16_t* off, int ch_words, int tid, int threads) {
+  const int khw = a.d.kh * a.d.kw;
+  for (int i = tid; i < a.n; i += threads) {
+    int c = i / khw, rs = i % khw;
+    off[i] = (uint16_t)(c * ch_words + (rs / a.d.kw) * a.pitch + (rs % a.d.kw));
+  }
+}
+
+// Stages the tile whose first input row/column is (h0, w0) of image `ximg`; out-of-image positions become 0.0.
+__device__ __forceinline__ void load_tile(const PatchArgs& a, const float* __restrict__ ximg, int h0, int w0,
+                                          float* tile, int ch_words, int tid, int threads) {
+  const int per_ch = a.in_h * a.in_w;
+  const int total = a.d.C * per_ch;
+  for (int idx = tid; idx < total; idx += threads) {
+    int c = a.magic_per_ch ? (int)__umulhi((unsigned)idx, a.magic_per_ch) : idx;  // magic 0: divisor 1
+    int rem = idx - c * per_ch;
+    int r = a.magic_in_w ? (int)__umulhi((unsigned)rem, a.magic_in_w) : rem;
+    int s = rem - r * a.in_w;
+    int h = h0 + r, w = w0 + s;
+    float v = 0.0f;
+    if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
+      v = __ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w);
+    tile[c * ch_words + r * a.pitch + s] = v;
+  }
+}
+
+struct TileCoord {
+  int img, ho0, wo0, h0, w0, th, tw;
+};
+
+__device__ __forceinline__ TileCoord tile_coord(const PatchArgs& a, int64_t tile_id) {
+  const int64_t tiles_per_img = (int64_t)a.tiles_h * a.tiles_w;
+  TileCoord t;
+  t.img = (int)(tile_id / tiles_per_img);
+  const int trem = (int)(tile_id % tiles_per_img);
+  t.ho0 = (trem / a.tiles_w) * a.TH;
+  t.wo0 = (trem % a.tiles_w) * a.TW;
+  t.h0 = t.ho0 * a.d.stride_h - a.d.pad_h;
+  t.w0 = t.wo0 * a.d.stride_w - a.d.pad_w;
+  t.th = min(a.TH, a.Ho - t.ho0);
+  t.tw = min(a.TW, a.Wo - t.wo0);
+  return t;
+}
+
+#ifndef DAB_WARP_MINBLOCKS
+#define DAB_WARP_MINBLOCKS 3  // CTAs per SM the one-warp-per-patch kernel is compiled for (register budget)
+#endif
+
+template <int R, bool kFull>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binarize_patches_warp_kernel(const PatchArgs a) {
+  constexpr int THREADS = kWarpsPerCta * 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* rcp = reinterpret_cast<double*>(smem_raw);
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + rcp_table_slots(a.n));
+  float* tile = reinterpret_cast<float*>(scratch_all + kWarpsPerCta * 32 * R);
+  const int ch_words = a.in_h * a.pitch;
+  uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* scratch = scratch_all + warp * (32 * R);
+  fill_reciprocals(rcp, a.n, threadIdx.x, THREADS);
+  fill_offsets(a, off, ch_words, threadIdx.x, THREADS);
+
+  const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+    const TileCoord t = tile_coord(a, tile_id);
+    __syncthreads();  // the previous tile is no longer read
+    load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
+    __syncthreads();
+
+    for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
+      const int lh = p / t.tw, lw = p % t.tw;
+      const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+      auto value = [origin, off](int i) { return origin[off[i]]; };
+      uint32_t kreg[R];
+      RowResult res = warp_code_row<R, kFull>(value, a.n, lane, scratch, rcp, kreg);
+      const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
+      if (lane == 0) {
+        a.pK[pi] = res.K;
+        a.pgamma[pi] = res.alpha;
+        a.pdelta[pi] = res.beta;
+        if (a.pflags) a.pflags[pi] = res.flags;
+      }
+      uint32_t mine = warp_mask_words<R, kFull>(kreg, a.n, lane, res);
+      uint32_t* mrow = a.pmask + pi * (int64_t)a.ldp;
+      for (int w = lane; w < a.ldp; w += 32) mrow[w] = (w < 32) ? mine : 0u;
+    }
+  }
+}
+
+template <int W, int WARPS, int R, bool kFull, bool kTable>
+__global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(const PatchArgs a) {
+  constexpr int G = WARPS / W;
+  constexpr int THREADS = WARPS * 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* rcp = reinterpret_cast<double*>(smem_raw);
+  GroupShared* gs_all = reinterpret_cast<GroupShared*>(rcp + (kTable ? rcp_table_slots(a.n) : 0));
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(gs_all + G);
+  float* tile = reinterpret_cast<float*>(scratch_all + (size_t)G * a.scratch_words);
+  const int ch_words = a.in_h * a.pitch;
+  uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
+
+  const int group = threadIdx.x / (32 * W);
+  const int tig = threadIdx.x % (32 * W);
+  GroupShared* gs = gs_all + group;
+  uint32_t* scratch = scratch_all + (size_t)group * a.scratch_words;
+  const int bar_id = 1 + group;
+  if (kTable) fill_reciprocals(rcp, a.n, threadIdx.x, THREADS);
+  fill_offsets(a, off, ch_words, threadIdx.x, THREADS);
+
+  const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+    const TileCoord t = tile_coord(a, tile_id);
+    __syncthreads();
+    load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
+    __syncthreads();
+
+    for (int p = group; p < t.th * t.tw; p += G) {
+      const int lh = p / t.tw, lw = p % t.tw;
+      const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+      auto value = [origin, off](int i) { return origin[off[i]]; };
+      uint32_t kreg[R];
+      group_code_row<W, R, kFull, kTable>(value, a.n, tig, scratch, gs, bar_id, rcp, kreg);
+      const RowResult res = gs->result;
+      const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
+      if (tig == 0) {
+        a.pK[pi] = res.K;
+        a.pgamma[pi] = res.alpha;
+        a.pdelta[pi] = res.beta;
+        if (a.pflags) a.pflags[pi] = res.flags;
+      }
+      group_store_mask<W, R, kFull>(kreg, a.n, a.ldp, tig, res, a.pmask + pi * (int64_t)a.ldp);
+      group_barrier(bar_id, 32 * W);
+    }
+  }
+}
+
+// Picks the tile: the largest of a few shapes whose staged input fits the shared-memory budget.
+static void choose_tile(const dab_conv_desc& d, int Ho, int Wo, size_t budget_bytes, PatchArgs* a) {
+  static const int shapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
+  for (auto& sh : shapes) {
+    int TH = sh[0] < Ho ? sh[0] : Ho, TW = sh[1] < Wo ? sh[1] : Wo;
+    int in_h = (TH - 1) * d.stride_h + d.kh, in_w = (TW - 1) * d.stride_w + d.kw;
+    int pitch = in_w | 1;  // odd pitch spreads the rows of a patch over the banks
+    size_t bytes = (size_t)d.C * in_h * pitch * sizeof(float);
+    if (bytes <= budget_bytes || (TH == 1 && TW == 1)) {
+      a->TH = TH; a->TW = TW; a->in_h = in_h; a->in_w = in_w; a->pitch = pitch;
+      a->tiles_h = (Ho + TH - 1) / TH; a->tiles_w = (Wo + TW - 1) / TW;
+      const uint64_t pc = (uint64_t)in_h * in_w, two32 = 0x100000000ull;
+      a->magic_per_ch = pc > 1 ? (uint32_t)((two32 + pc - 1) / pc) : 0u;
+      a->magic_in_w = in_w > 1 ? (uint32_t)((two32 + (uint64_t)in_w - 1) / (uint64_t)in_w) : 0u;
+      return;
+    }
+  }
+}
+
+template <typename Kernel>
+static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes, int threads, cudaStream_t stream) {
+  const size_t limit = 200 * 1024;
+  size_t budget = limit > fixed_bytes ? limit - fixed_bytes : 0;
+  if (budget > 72 * 1024) budget = 72 * 1024;  // leave room for more than one CTA per SM when the tile is small
+  choose_tile(a.d, a.Ho, a.Wo, budget, &a);
+  size_t tile_words = (size_t)a.d.C * a.in_h * a.pitch;
+  if (tile_words > 65535) return cudaErrorInvalidValue;  // offsets are 16-bit
+  size_t smem = fixed_bytes + tile_words * sizeof(float) + sizeof(uint16_t) * a.n + 16;
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int64_t tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  int64_t blocks = tiles < 148 * 8 ? tiles : 148 * 8;
+  kern<<<(unsigned)blocks, threads, smem, stream>>>(a);
+  return cudaGetLastError();
+}
+
+template <int R, bool kFull>
+static cudaError_t launch_patches_warp(PatchArgs& a, cudaStream_t stream) {
+  size_t fixed = sizeof(double) * rcp_table_slots(a.n) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
+  return launch_patches(binarize_patches_warp_kernel<R, kFull>, a, fixed, kWarpsPerCta * 32, stream);
+}
+
+template <int W, int WARPS, int R, bool kFull, bool kTable>
+static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream) {
+  constexpr int G = WARPS / W;
+  a.scratch_words = scratch_words_for(a.n, W);
+  size_t fixed = (kTable ? sizeof(double) * rcp_table_slots(a.n) : 0) + sizeof(GroupShared) * G +
+                 sizeof(uint32_t) * (size_t)a.scratch_words * G;
+  return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, stream);
+}
+
+cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
+                                    float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
+                                    cudaStream_t stream) {
+  PatchArgs a;
+  a.d = d; a.Ho = Ho; a.Wo = Wo; a.n = d.C * d.kh * d.kw;
+  a.scratch_words = 0;
+  a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
+  if (a.n == 256) return launch_patches_warp<8, true>(a, stream);
+  if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
+#ifdef DAB_EXP_576_GROUP
+  if (a.n == 576) return launch_patches_group<2, 8, 9, true, true>(a, stream);
+#endif
+  if (a.n == 576) return launch_patches_warp<18, true>(a, stream);
+  if (a.n <= 576) return launch_patches_warp<18, false>(a, stream);
+  if (a.n == 1024) return launch_patches_warp<32, true>(a, stream);
+  if (a.n <= 1024) return launch_patches_warp<32, false>(a, stream);
+  if (a.n == 1152) return launch_patches_group<2, 8, 18, true, true>(a, stream);
+  if (a.n <= 2048) return launch_patches_group<2, 8, 32, false, true>(a, stream);
+  if (a.n == 2304) return launch_patches_group<4, 8, 18, true, true>(a, stream);
+  if (a.n <= 4096) return launch_patches_group<4, 8, 32, false, true>(a, stream);
+  if (a.n == 4608) return launch_patches_group<8, 8, 18, true, true>(a, stream);
+  if (a.n <= 8192) return launch_patches_group<8, 8, 32, false, true>(a, stream);
+  if (a.n == 9216) return launch_patches_group<16, 16, 18, true, false>(a, stream);
+  return launch_patches_group<16, 16, 32, false, false>(a, stream);
+}
+
+}  // namespace dab

@@ -22,7 +22,15 @@
 
 namespace dab {
 
+constexpr int kWarpsPerCta = 8;             // warps of a CTA in the one-warp-per-row kernels
 constexpr uint32_t kZeroKey = 0x80000000u;  // order_key(0.0f)
+
+// Scratch words a group of W warps needs for rows of up to n values (the largest sort capacity reachable).
+inline int scratch_words_for(int n, int W) {
+  int cap = 128 * W;
+  while (cap < n) cap <<= 1;
+  return cap;
+}
 constexpr double kBand = 1.0 - 1e-13;       // splits whose approximate objective is below max*kBand cannot win
 
 __device__ __forceinline__ void group_barrier(int bar_id, int threads) {
