@@ -164,40 +164,47 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
   }
 }
 
-// Picks the tile: the largest of a few shapes whose staged input fits the shared-memory budget.
-static void choose_tile(const dab_conv_desc& d, int Ho, int Wo, size_t budget_bytes, PatchArgs* a) {
-  static const int shapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
-  for (auto& sh : shapes) {
-    int TH = sh[0] < Ho ? sh[0] : Ho, TW = sh[1] < Wo ? sh[1] : Wo;
-    int in_h = (TH - 1) * d.stride_h + d.kh, in_w = (TW - 1) * d.stride_w + d.kw;
-    int pitch = in_w | 1;  // odd pitch spreads the rows of a patch over the banks
-    size_t bytes = (size_t)d.C * in_h * pitch * sizeof(float);
-    if (bytes <= budget_bytes || (TH == 1 && TW == 1)) {
-      a->TH = TH; a->TW = TW; a->in_h = in_h; a->in_w = in_w; a->pitch = pitch;
-      a->tiles_h = (Ho + TH - 1) / TH; a->tiles_w = (Wo + TW - 1) / TW;
-      const uint64_t pc = (uint64_t)in_h * in_w, two32 = 0x100000000ull;
-      a->magic_per_ch = pc > 1 ? (uint32_t)((two32 + pc - 1) / pc) : 0u;
-      a->magic_in_w = in_w > 1 ? (uint32_t)((two32 + (uint64_t)in_w - 1) / (uint64_t)in_w) : 0u;
-      return;
-    }
-  }
+// Tile shapes tried, largest first.
+static const int kTileShapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
+
+static void set_tile(const dab_conv_desc& d, int Ho, int Wo, const int (&sh)[2], PatchArgs* a) {
+  int TH = sh[0] < Ho ? sh[0] : Ho, TW = sh[1] < Wo ? sh[1] : Wo;
+  int in_h = (TH - 1) * d.stride_h + d.kh, in_w = (TW - 1) * d.stride_w + d.kw;
+  a->TH = TH; a->TW = TW; a->in_h = in_h; a->in_w = in_w;
+  a->pitch = in_w | 1;  // odd pitch spreads the rows of a patch over the banks
+  a->tiles_h = (Ho + TH - 1) / TH; a->tiles_w = (Wo + TW - 1) / TW;
+  const uint64_t pc = (uint64_t)in_h * in_w, two32 = 0x100000000ull;
+  a->magic_per_ch = pc > 1 ? (uint32_t)((two32 + pc - 1) / pc) : 0u;
+  a->magic_in_w = in_w > 1 ? (uint32_t)((two32 + (uint64_t)in_w - 1) / (uint64_t)in_w) : 0u;
 }
 
+// Picks the tile and launches.  The largest tile is taken that still lets at least 16 warps be resident per SM
+// (shared memory is the limit); if no shape reaches that, the shape with the most resident CTAs wins.
 template <typename Kernel>
 static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes, int threads, cudaStream_t stream) {
-  const size_t limit = 200 * 1024;
-  size_t budget = limit > fixed_bytes ? limit - fixed_bytes : 0;
-  if (budget > 72 * 1024) budget = 72 * 1024;  // leave room for more than one CTA per SM when the tile is small
-  choose_tile(a.d, a.Ho, a.Wo, budget, &a);
-  size_t tile_words = (size_t)a.d.C * a.in_h * a.pitch;
-  if (tile_words > 65535) return cudaErrorInvalidValue;  // offsets are 16-bit
-  size_t smem = fixed_bytes + tile_words * sizeof(float) + sizeof(uint16_t) * a.n + 16;
-  if (smem > 227 * 1024) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t sm_bytes = 228 * 1024, cta_reserve = 1024, cta_limit = 227 * 1024;
+  const int want_ctas = (16 * 32 + threads - 1) / threads;
+  int best = -1, best_ctas = 0;
+  size_t best_smem = 0;
+  for (int i = 0; i < (int)(sizeof(kTileShapes) / sizeof(kTileShapes[0])); ++i) {
+    PatchArgs t = a;
+    set_tile(a.d, a.Ho, a.Wo, kTileShapes[i], &t);
+    size_t tile_words = (size_t)a.d.C * t.in_h * t.pitch;
+    if (tile_words > 65535) continue;  // offsets are 16-bit
+    size_t smem = fixed_bytes + tile_words * sizeof(float) + sizeof(uint16_t) * a.n + 16;
+    if (smem > cta_limit) continue;
+    int ctas = (int)(sm_bytes / (smem + cta_reserve));
+    if (ctas > 2048 / threads) ctas = 2048 / threads;
+    if (ctas > best_ctas) { best = i; best_ctas = ctas; best_smem = smem; }
+    if (ctas >= want_ctas) break;
+  }
+  if (best < 0) return cudaErrorInvalidValue;
+  set_tile(a.d, a.Ho, a.Wo, kTileShapes[best], &a);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)best_smem);
   if (e != cudaSuccess) return e;
   int64_t tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
   int64_t blocks = tiles < 148 * 8 ? tiles : 148 * 8;
-  kern<<<(unsigned)blocks, threads, smem, stream>>>(a);
+  kern<<<(unsigned)blocks, threads, best_smem, stream>>>(a);
   return cudaGetLastError();
 }
 
@@ -225,9 +232,6 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
   if (a.n == 256) return launch_patches_warp<8, true>(a, stream);
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
-#ifdef DAB_EXP_576_GROUP
-  if (a.n == 576) return launch_patches_group<2, 8, 9, true, true>(a, stream);
-#endif
   if (a.n == 576) return launch_patches_warp<18, true>(a, stream);
   if (a.n <= 576) return launch_patches_warp<18, false>(a, stream);
   if (a.n == 1024) return launch_patches_warp<32, true>(a, stream);
@@ -236,8 +240,8 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   if (a.n <= 2048) return launch_patches_group<2, 8, 32, false, true>(a, stream);
   if (a.n == 2304) return launch_patches_group<4, 8, 18, true, true>(a, stream);
   if (a.n <= 4096) return launch_patches_group<4, 8, 32, false, true>(a, stream);
-  if (a.n == 4608) return launch_patches_group<8, 8, 18, true, true>(a, stream);
-  if (a.n <= 8192) return launch_patches_group<8, 8, 32, false, true>(a, stream);
+  if (a.n == 4608) return launch_patches_group<8, 16, 18, true, true>(a, stream);
+  if (a.n <= 8192) return launch_patches_group<8, 16, 32, false, true>(a, stream);
   if (a.n == 9216) return launch_patches_group<16, 16, 18, true, false>(a, stream);
   return launch_patches_group<16, 16, 32, false, false>(a, stream);
 }
