@@ -114,21 +114,16 @@ cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_
                             float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
                             cudaStream_t stream) {
 #define DAB_ARGS values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream
+  // A matrix may have few rows (a layer's filters), so a row gets enough warps for at most 8 keys per thread
+  // even when none of its values is zero: short critical path per row, and the 8-key network is the most
+  // efficient one per element.
   if (n == 256) return launch_rows_warp<8, true>(DAB_ARGS);
   if (n <= 256) return launch_rows_warp<8, false>(DAB_ARGS);
-  if (n == 576) return launch_rows_warp<18, true>(DAB_ARGS);
-  if (n <= 576) return launch_rows_warp<18, false>(DAB_ARGS);
-  if (n == 1024) return launch_rows_warp<32, true>(DAB_ARGS);
-  if (n <= 1024) return launch_rows_warp<32, false>(DAB_ARGS);
-  // rows of exactly 576 values per warp (1152, 2304, 4608, 9216) get the variant without bounds tests
-  if (n == 1152) return launch_rows_group<2, 8, 18, true, true>(DAB_ARGS);
-  if (n <= 2048) return launch_rows_group<2, 8, 32, false, true>(DAB_ARGS);
-  if (n == 2304) return launch_rows_group<4, 8, 18, true, true>(DAB_ARGS);
-  if (n <= 4096) return launch_rows_group<4, 8, 32, false, true>(DAB_ARGS);
-  if (n == 4608) return launch_rows_group<8, 8, 18, true, true>(DAB_ARGS);
-  if (n <= 8192) return launch_rows_group<8, 8, 32, false, true>(DAB_ARGS);
-  if (n == 9216) return launch_rows_group<16, 16, 18, true, false>(DAB_ARGS);
-  return launch_rows_group<16, 16, 32, false, false>(DAB_ARGS);
+  if (n <= 1024) return launch_rows_group<4, 8, 8, false, true>(DAB_ARGS);
+  if (n <= 2048) return launch_rows_group<8, 8, 8, false, true>(DAB_ARGS);
+  if (n <= 4096) return launch_rows_group<16, 16, 8, false, true>(DAB_ARGS);
+  if (n <= 8192) return launch_rows_group<32, 32, 8, false, true>(DAB_ARGS);
+  return launch_rows_group<32, 32, 16, false, false>(DAB_ARGS);
 #undef DAB_ARGS
 }
 

@@ -127,17 +127,17 @@ struct RowResult {
 };
 
 struct GroupShared {   // per group of more than one warp, in shared memory
-  double wsum[16];     // per-warp sums
-  double wmax[16];     // per-warp maxima of the approximate objective
-  int wneg[16];        // per-warp counts of negative keys
-  uint32_t wfirst[17]; // first key of each warp (index W: pad key)
-  long long wbestD[16];
-  int wbestS[16];
-  double wbestP[16];
-  uint32_t wbestT[16];
-  int wcnt[16];        // per-warp counts of non-zero keys
-  uint32_t wkmin[16];  // per-warp smallest and largest key
-  uint32_t wkmax[16];
+  double wsum[32];     // per-warp sums
+  double wmax[32];     // per-warp maxima of the approximate objective
+  int wneg[32];        // per-warp counts of negative keys
+  uint32_t wfirst[33]; // first key of each warp (index W: pad key)
+  long long wbestD[32];
+  int wbestS[32];
+  double wbestP[32];
+  uint32_t wbestT[32];
+  int wcnt[32];        // per-warp counts of non-zero keys
+  uint32_t wkmin[32];  // per-warp smallest and largest key
+  uint32_t wkmax[32];
   RowResult result;
 };
 
