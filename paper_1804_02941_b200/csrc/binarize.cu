@@ -117,7 +117,6 @@ cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_
   // A matrix may have few rows (a layer's filters), so a row gets enough warps for at most 8 keys per thread
   // even when none of its values is zero: short critical path per row, and the 8-key network is the most
   // efficient one per element.
-  if (n == 256) return launch_rows_warp<8, true>(DAB_ARGS);
   if (n <= 256) return launch_rows_warp<8, false>(DAB_ARGS);
   if (n <= 1024) return launch_rows_group<4, 8, 8, false, true>(DAB_ARGS);
   if (n <= 2048) return launch_rows_group<8, 8, 8, false, true>(DAB_ARGS);

@@ -230,18 +230,19 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   a.d = d; a.Ho = Ho; a.Wo = Wo; a.n = d.C * d.kh * d.kw;
   a.scratch_words = 0;
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
-  if (a.n == 256) return launch_patches_warp<8, true>(a, stream);
+  // The patch lengths of the common 3x3 layers (576 values per warp) have variants without bounds tests whose
+  // group size suits rows that are at least half zeros.  Any other length gets enough warps for at most 16
+  // values per thread, so that rows with up to half their values non-zero sort with 8 keys per thread.
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
   if (a.n == 576) return launch_patches_warp<18, true>(a, stream);
   if (a.n <= 576) return launch_patches_warp<18, false>(a, stream);
-  if (a.n == 1024) return launch_patches_warp<32, true>(a, stream);
-  if (a.n <= 1024) return launch_patches_warp<32, false>(a, stream);
+  if (a.n <= 1024) return launch_patches_group<2, 8, 16, false, true>(a, stream);
   if (a.n == 1152) return launch_patches_group<2, 8, 18, true, true>(a, stream);
-  if (a.n <= 2048) return launch_patches_group<2, 8, 32, false, true>(a, stream);
+  if (a.n <= 2048) return launch_patches_group<4, 8, 16, false, true>(a, stream);
   if (a.n == 2304) return launch_patches_group<4, 8, 18, true, true>(a, stream);
-  if (a.n <= 4096) return launch_patches_group<4, 8, 32, false, true>(a, stream);
+  if (a.n <= 4096) return launch_patches_group<8, 16, 16, false, true>(a, stream);
   if (a.n == 4608) return launch_patches_group<8, 16, 18, true, true>(a, stream);
-  if (a.n <= 8192) return launch_patches_group<8, 16, 32, false, true>(a, stream);
+  if (a.n <= 8192) return launch_patches_group<16, 16, 16, false, true>(a, stream);
   if (a.n == 9216) return launch_patches_group<16, 16, 18, true, false>(a, stream);
   return launch_patches_group<16, 16, 32, false, false>(a, stream);
 }

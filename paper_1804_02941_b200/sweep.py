@@ -1,0 +1,145 @@
+"""Stage-by-stage timings of libdab on the five synthetic workload configurations.
+
+`python -m paper_1804_02941_b200.sweep [--configs 1,2,3,4,5] [--batch5 256]` prints one JSON line per
+(config, layer or point, stage): device time by CUDA events (best of a few repetitions after warm-up), the
+stage's throughput and its fraction of the relevant roofline (HBM copy bandwidth for binarize and pack, the
+population-count rate for the contraction).  bench.py is the benchmark of record; this is the wider table.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+import dab_synth
+from dab_synth import configs
+import paper_1804_02941_b200 as dab
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SM_COUNT, POPC_PER_CLK, WORDS_PER_POPC = 148, 16, 1.5
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+def timed(fn, reps=5, warm=2):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    return best
+
+
+def emit(**kw):
+    print(json.dumps(kw), flush=True)
+
+
+def conv_layer(cfg, L, stream, hbm, tops_peak, dense=False):
+    dev = torch.device("cuda")
+    x = torch.from_numpy(L.inputs(stream=stream, dense=dense)).to(dev)
+    w = torch.from_numpy(L.weights(stream=stream)).to(dev)
+    wd = dab.dab_binarize(w)
+    desc = dab.make_desc(L.x_shape(), L.Cout, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad))
+    P, ld = L.patches, dab.dab_default_ld(L.n)
+    pK = torch.empty(P, dtype=torch.int32, device=dev)
+    pg, pd = torch.empty(P, device=dev), torch.empty(P, device=dev)
+    pm = torch.empty((P, ld), dtype=torch.int32, device=dev)
+    y = torch.empty((L.N, L.Cout, L.Ho, L.Wo), device=dev)
+    t_w = timed(lambda: dab.dab_binarize_into(w, wd.K, wd.alpha, wd.beta, wd.mask, wd.flags))
+    t_p = timed(lambda: dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, None))
+    t_c = timed(lambda: dab.dab_binary_conv_contract(desc, pm, pK, pg, pd, wd, y, None))
+    wd_words = dab.dab_words_per_row(L.n)
+    bytes_p = 4 * x.numel() + P * (4 * wd_words + 12)
+    bytes_w = L.Cout * (4 * L.n + 4 * wd_words + 12)
+    common = dict(config=cfg, layer=L.name, n=L.n, patches=P, filters=L.Cout, inputs="dense" if dense else "relu60")
+    emit(stage="binarize_filters", ms=t_w, gbs=bytes_w / t_w / 1e6, hbm_frac=bytes_w / t_w / 1e6 / hbm, **common)
+    emit(stage="binarize_patches", ms=t_p, gbs=bytes_p / t_p / 1e6, hbm_frac=bytes_p / t_p / 1e6 / hbm, **common)
+    emit(stage="contract", ms=t_c, tops_equiv=L.binary_ops / t_c / 1e9, alu_frac=L.binary_ops / t_c / 1e9 / tops_peak,
+         **common)
+    emit(stage="conv_total", ms=t_p + t_c, tops_equiv=L.binary_ops / (t_p + t_c) / 1e9, **common)
+
+
+def gemm_point(m, k, hbm, tops_peak):
+    dev = torch.device("cuda")
+    A, B = configs.config3_operands(m, k)
+    Ad, Bd = torch.from_numpy(A).to(dev), torch.from_numpy(B).to(dev)
+    a, b = dab.dab_binarize(Ad), dab.dab_binarize(Bd)
+    Cm = torch.empty((m, m), device=dev)
+    t_b = timed(lambda: dab.dab_binarize_into(Ad, a.K, a.alpha, a.beta, a.mask, a.flags))
+    t_g = timed(lambda: dab.dab_binary_gemm(a, b, out=Cm))
+    wdw = dab.dab_words_per_row(k)
+    bytes_b = m * (4 * k + 4 * wdw + 12)
+    ops = 2 * m * m * k
+    emit(config=3, stage="binarize", M=m, n=k, ms=t_b, gbs=bytes_b / t_b / 1e6, hbm_frac=bytes_b / t_b / 1e6 / hbm,
+         inputs="laplace dense")
+    emit(config=3, stage="gemm", M=m, N=m, n=k, ms=t_g, tops_equiv=ops / t_g / 1e9, alu_frac=ops / t_g / 1e9 / tops_peak,
+         store_gbs=4 * m * m / t_g / 1e6)
+
+
+def pack_point(rows, n, hbm):
+    dev = torch.device("cuda")
+    bits = (torch.rand((rows, n), device=dev) < 0.4).to(torch.uint8)
+    ld = dab.dab_default_ld(n)
+    mask = torch.empty((rows, ld), dtype=torch.int32, device=dev)
+    K = torch.empty(rows, dtype=torch.int32, device=dev)
+    import ctypes as C
+    L = dab.lib()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    fn = lambda: L.dab_pack(C.c_void_p(bits.data_ptr()), rows, n, n, C.c_void_p(mask.data_ptr()), ld,
+                            C.c_void_p(K.data_ptr()), st)
+    t = timed(fn)
+    b = rows * (n + 4 * dab.dab_words_per_row(n) + 4)
+    emit(stage="pack", rows=rows, n=n, ms=t, gbs=b / t / 1e6, hbm_frac=b / t / 1e6 / hbm)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="1,2,3,4,5")
+    ap.add_argument("--batch5", type=int, default=256)
+    args = ap.parse_args()
+    want = set(args.configs.split(","))
+    hbm, mhz, src = peaks()
+    tops_peak = POPC_PER_CLK * WORDS_PER_POPC * SM_COUNT * mhz * 1e6 * 64 / 1e12
+    emit(peaks=dict(hbm_gbs=hbm, source=src, contraction_tops_equiv=tops_peak,
+                    contraction_peak="16 popc/clk/SM x 1.5 words/popc x 148 SMs x %.0f MHz x 64" % mhz))
+    if "1" in want:
+        conv_layer(1, configs.config1()[0], 0, hbm, tops_peak)
+    if "2" in want:
+        for i, L in enumerate(configs.config2()):
+            conv_layer(2, L, i, hbm, tops_peak)
+    if "3" in want:
+        for m, k in configs.CONFIG3_POINTS:
+            gemm_point(m, k, hbm, tops_peak)
+        pack_point(65536, 4608, hbm)
+        pack_point(802816, 576, hbm)
+    if "4" in want:
+        for i, L in enumerate(configs.config4()):
+            conv_layer(4, L, 20 + i, hbm, tops_peak)
+    if "5" in want:
+        seen = set()
+        for i, L in enumerate(configs.config5(args.batch5)):
+            key = (L.C, L.H, L.Cout, L.stride)
+            if key in seen:
+                continue
+            seen.add(key)
+            conv_layer(5, L, i, hbm, tops_peak)
+        conv_layer(5, configs.config5(args.batch5)[0], 50, hbm, tops_peak, dense=True)
+
+
+if __name__ == "__main__":
+    main()
