@@ -5,46 +5,67 @@ namespace dab {
 
 // Four bytes in one word -> 4 bits (bit k set iff byte k is non-zero).
 __device__ __forceinline__ uint32_t nibble_of(uint32_t x) {
-  uint32_t t = (((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x) & 0x80808080u;  // bit 7 of each non-zero byte
-  return (((t >> 7) * 0x00204081u) >> 21) & 0xFu;
+  // bit 7 of every non-zero byte: adding 0x7F to the low seven bits carries into bit 7 unless they are all 0
+  const uint32_t t = (((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x) & 0x80808080u;
+  // bits 7, 15, 23, 31 -> bits 28..31: the partial products of this multiplier land on distinct bits (no carries)
+  return (t * 0x00204081u) >> 28;
 }
 
-// Fast path: rows start on 16-byte boundaries.  A thread turns 16 bytes into 16 bits; a lane pair makes a word.
+__device__ __forceinline__ uint32_t bits16_of(uint4 q) {
+  return nibble_of(q.x) | (nibble_of(q.y) << 4) | (nibble_of(q.z) << 8) | (nibble_of(q.w) << 12);
+}
+
+// Fast path: rows start on 16-byte boundaries.  Work is laid out flat over (row, word): a thread turns 32 bytes
+// into one word, so all lanes stay busy however short the rows are.  Pad words come out as 0.
+// magic = floor(2^32 / ld_mask) gives the row of a flat index with one multiply and one correction.
 __global__ void __launch_bounds__(256) pack_aligned_kernel(const uint8_t* __restrict__ bits, int64_t rows, int32_t n,
                                                            int64_t ld_bits, uint32_t* __restrict__ mask,
-                                                           int32_t ld_mask, int32_t* __restrict__ K) {
+                                                           int32_t ld_mask, uint32_t magic, int64_t row_begin) {
+  const uint32_t total = (uint32_t)rows * (uint32_t)ld_mask;  // the host keeps this below 2^31 per launch
+  for (uint32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+    uint32_t row = __umulhi(t, magic);
+    uint32_t w = t - row * (uint32_t)ld_mask;
+    if (w >= (uint32_t)ld_mask) { w -= ld_mask; ++row; }
+    const int e0 = (int)w * 32;
+    const uint8_t* b = bits + (row_begin + row) * ld_bits + e0;
+    uint32_t word = 0;
+    if (e0 + 32 <= n) {
+      const uint4 q0 = __ldg(reinterpret_cast<const uint4*>(b));
+      const uint4 q1 = __ldg(reinterpret_cast<const uint4*>(b) + 1);
+      word = bits16_of(q0) | (bits16_of(q1) << 16);
+    } else if (e0 < n) {  // the one ragged word of a row; words past the row stay 0
+      for (int k = 0; k < n - e0; ++k)
+        if (b[k]) word |= 1u << k;
+    }
+    mask[(row_begin + row) * (int64_t)ld_mask + w] = word;
+  }
+}
+
+// Ones per row from the packed words (second, small pass over 1/8 byte per element): a thread per row for
+// short rows (128-bit loads, every fetched sector fully used), a warp per row for long ones.
+__global__ void __launch_bounds__(256) count_ones_thread_kernel(const uint32_t* __restrict__ mask, int64_t rows,
+                                                                int32_t ld_mask, int32_t* __restrict__ K) {
+  for (int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; row < rows; row += (int64_t)gridDim.x * blockDim.x) {
+    const uint4* m = reinterpret_cast<const uint4*>(mask + row * (int64_t)ld_mask);
+    int c = 0;
+    for (int q = 0; q < ld_mask / 4; ++q) {
+      const uint4 v = __ldg(m + q);
+      c += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+    }
+    K[row] = c;
+  }
+}
+
+__global__ void __launch_bounds__(256) count_ones_warp_kernel(const uint32_t* __restrict__ mask, int64_t rows,
+                                                              int32_t ld_mask, int32_t* __restrict__ K) {
   const int lane = threadIdx.x & 31;
-  const int warps_per_block = blockDim.x >> 5;
-  const int64_t warp0 = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-  const int64_t warp_stride = (int64_t)gridDim.x * warps_per_block;
-  for (int64_t row = warp0; row < rows; row += warp_stride) {
-    const uint8_t* b = bits + row * ld_bits;
-    uint32_t* m = mask + row * (int64_t)ld_mask;
-    int count = 0;
-    // one pass of the warp covers 512 elements = 16 words
-    for (int w0 = 0; w0 < ld_mask; w0 += 16) {
-      int e0 = w0 * 32 + lane * 16;
-      uint32_t half = 0;
-      if (e0 + 16 <= n) {
-        uint4 q = *reinterpret_cast<const uint4*>(b + e0);
-        half = nibble_of(q.x) | (nibble_of(q.y) << 4) | (nibble_of(q.z) << 8) | (nibble_of(q.w) << 12);
-      } else {
-        for (int k = 0; k < 16; ++k)
-          if (e0 + k < n && b[e0 + k]) half |= 1u << k;
-      }
-      uint32_t other = __shfl_down_sync(0xFFFFFFFFu, half, 1);
-      uint32_t word = half | (other << 16);
-      int w = w0 + (lane >> 1);
-      if ((lane & 1) == 0 && w < ld_mask) {
-        m[w] = word;
-        count += __popc(word);
-      }
-    }
-    if (K) {
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) count += __shfl_down_sync(0xFFFFFFFFu, count, off);
-      if (lane == 0) K[row] = count;
-    }
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t row = warp0; row < rows; row += nwarps) {
+    int c = 0;
+    for (int w = lane; w < ld_mask; w += 32) c += __popc(mask[row * (int64_t)ld_mask + w]);
+    c = __reduce_add_sync(0xFFFFFFFFu, c);
+    if (lane == 0) K[row] = c;
   }
 }
 
@@ -77,9 +98,25 @@ cudaError_t launch_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld
   int64_t blocks = (rows + wpb - 1) / wpb;
   if (blocks > 148 * 64) blocks = 148 * 64;
   bool aligned = (reinterpret_cast<uintptr_t>(bits) % 16 == 0) && (ld_bits % 16 == 0);
-  if (aligned)
-    pack_aligned_kernel<<<(unsigned)blocks, threads, 0, stream>>>(bits, rows, n, ld_bits, mask, ld_mask, K);
-  else
+  if (aligned) {
+    const uint32_t magic = (uint32_t)(0x100000000ull / (uint64_t)ld_mask);  // ld_mask >= 4
+    const int64_t rows_per_launch = (int64_t)0x7FFFFFFF / ld_mask;
+    for (int64_t r0 = 0; r0 < rows; r0 += rows_per_launch) {
+      const int64_t nr = rows - r0 < rows_per_launch ? rows - r0 : rows_per_launch;
+      int64_t pb = (nr * ld_mask + threads - 1) / threads;
+      if (pb > 148 * 32) pb = 148 * 32;
+      pack_aligned_kernel<<<(unsigned)pb, threads, 0, stream>>>(bits, nr, n, ld_bits, mask, ld_mask, magic, r0);
+    }
+    if (K) {
+      if (ld_mask <= 64) {
+        int64_t cb = (rows + threads - 1) / threads;
+        if (cb > 148 * 32) cb = 148 * 32;
+        count_ones_thread_kernel<<<(unsigned)cb, threads, 0, stream>>>(mask, rows, ld_mask, K);
+      } else {
+        count_ones_warp_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mask, rows, ld_mask, K);
+      }
+    }
+  } else
     pack_bytes_kernel<<<(unsigned)blocks, threads, 0, stream>>>(bits, rows, n, ld_bits, mask, ld_mask, K);
   return cudaGetLastError();
 }
