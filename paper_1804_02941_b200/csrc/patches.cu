@@ -17,6 +17,9 @@ struct PatchArgs {
   int32_t pitch;           // words per staged row (>= in_w)
   int32_t tiles_h, tiles_w;
   int32_t scratch_words;
+  int32_t defer_dense;     // one-warp kernel: leave tiles that look dense to a second kernel (marks them in pK)
+  int32_t marked_only;     // group kernel: code only the tiles marked by the one-warp kernel
+  int32_t tile_shape;      // index into kTileShapes forced by the caller, -1: choose
   uint32_t magic_per_ch, magic_in_w;  // ceil(2^32 / d) for d = in_h*in_w and in_w: floor(i/d) = umulhi(i, magic); 0 if d == 1
   const float* x;
   int32_t* pK;
@@ -36,10 +39,12 @@ __device__ __forceinline__ void fill_offsets(const PatchArgs& a, uint16_t* off, 
 }
 
 // Stages the tile whose first input row/column is (h0, w0) of image `ximg`; out-of-image positions become 0.0.
-__device__ __forceinline__ void load_tile(const PatchArgs& a, const float* __restrict__ ximg, int h0, int w0,
-                                          float* tile, int ch_words, int tid, int threads) {
+// Returns the number of non-zero values this thread staged.
+__device__ __forceinline__ int load_tile(const PatchArgs& a, const float* __restrict__ ximg, int h0, int w0,
+                                         float* tile, int ch_words, int tid, int threads) {
   const int per_ch = a.in_h * a.in_w;
   const int total = a.d.C * per_ch;
+  int nonzero = 0;
   for (int idx = tid; idx < total; idx += threads) {
     int c = a.magic_per_ch ? (int)__umulhi((unsigned)idx, a.magic_per_ch) : idx;  // magic 0: divisor 1
     int rem = idx - c * per_ch;
@@ -50,8 +55,14 @@ __device__ __forceinline__ void load_tile(const PatchArgs& a, const float* __res
     if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
       v = __ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w);
     tile[c * ch_words + r * a.pitch + s] = v;
+    nonzero += (v != 0.0f);
   }
+  return nonzero;
 }
+
+// Index of the first patch of a tile: where the one-warp kernel leaves its "dense tile" mark (K = -1, a value no
+// coded patch has) for the group kernel that follows it on the stream.
+constexpr int32_t kDenseMark = -1;
 
 struct TileCoord {
   int img, ho0, wo0, h0, w0, th, tw;
@@ -85,6 +96,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
   const int ch_words = a.in_h * a.pitch;
   uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
 
+  __shared__ int tile_nonzero;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t* scratch = scratch_all + warp * (32 * R);
   fill_reciprocals(rcp, a.n, threadIdx.x, THREADS);
@@ -94,8 +106,26 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
     __syncthreads();  // the previous tile is no longer read
-    load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
-    __syncthreads();
+    if (threadIdx.x == 0) tile_nonzero = 0;
+    int nz = load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x,
+                       THREADS);
+    const int64_t first_patch = ((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0;
+    if (a.defer_dense) {
+      // One warp per patch suits patches whose non-zero values fit 8 keys per lane (at most 256).  A tile whose
+      // density says otherwise (expected non-zeros per patch = density of the staged region * n > 256) is left to
+      // the group kernel, which sorts it with about 8 keys per thread again.
+      __syncthreads();
+      nz = __reduce_add_sync(0xFFFFFFFFu, nz);
+      if (lane == 0 && nz) atomicAdd(&tile_nonzero, nz);
+      __syncthreads();
+      const int64_t staged = (int64_t)a.d.C * a.in_h * a.in_w;
+      if ((int64_t)tile_nonzero * a.n > 256 * staged) {
+        if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+        continue;
+      }
+    } else {
+      __syncthreads();
+    }
 
     for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
       const int lh = p / t.tw, lw = p % t.tw;
@@ -140,6 +170,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
   const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
+    if (a.marked_only && a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] != kDenseMark) continue;
     __syncthreads();
     load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
     __syncthreads();
@@ -187,6 +218,7 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
   int best = -1, best_ctas = 0;
   size_t best_smem = 0;
   for (int i = 0; i < (int)(sizeof(kTileShapes) / sizeof(kTileShapes[0])); ++i) {
+    if (a.tile_shape >= 0 && i != a.tile_shape) continue;
     PatchArgs t = a;
     set_tile(a.d, a.Ho, a.Wo, kTileShapes[i], &t);
     size_t tile_words = (size_t)a.d.C * t.in_h * t.pitch;
@@ -199,6 +231,7 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
     if (ctas >= want_ctas) break;
   }
   if (best < 0) return cudaErrorInvalidValue;
+  a.tile_shape = best;
   set_tile(a.d, a.Ho, a.Wo, kTileShapes[best], &a);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)best_smem);
   if (e != cudaSuccess) return e;
@@ -229,13 +262,20 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   PatchArgs a;
   a.d = d; a.Ho = Ho; a.Wo = Wo; a.n = d.C * d.kh * d.kw;
   a.scratch_words = 0;
+  a.defer_dense = 0; a.marked_only = 0; a.tile_shape = -1;
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
   // The patch lengths of the common 3x3 layers (576 values per warp) have variants without bounds tests whose
   // group size suits rows that are at least half zeros.  Any other length gets enough warps for at most 16
   // values per thread, so that rows with up to half their values non-zero sort with 8 keys per thread.
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
-  if (a.n == 576) return launch_patches_warp<18, true>(a, stream);
-  if (a.n <= 576) return launch_patches_warp<18, false>(a, stream);
+  if (a.n > 256 && a.n <= 576) {
+    // first the one-warp kernel on the tiles it suits, then four warps per patch on the tiles it marked as dense
+    a.defer_dense = 1;
+    cudaError_t e = a.n == 576 ? launch_patches_warp<18, true>(a, stream) : launch_patches_warp<18, false>(a, stream);
+    if (e != cudaSuccess) return e;
+    a.defer_dense = 0; a.marked_only = 1;  // a.tile_shape now holds the first kernel's tile
+    return launch_patches_group<4, 8, 5, false, true>(a, stream);
+  }
   if (a.n <= 1024) return launch_patches_group<2, 8, 16, false, true>(a, stream);
   if (a.n == 1152) return launch_patches_group<2, 8, 18, true, true>(a, stream);
   if (a.n <= 2048) return launch_patches_group<4, 8, 16, false, true>(a, stream);

@@ -205,6 +205,16 @@ def test_conv_on_stroke_image_patches(dab):
     _check_conv(dab, x, w, 5, 5, (1, 1), (2, 2))
 
 
+def test_conv_with_dense_and_sparse_regions(dab):
+    # n = 576: tiles whose staged values are mostly non-zero are coded by four warps per patch, the others by one
+    # warp per patch; an image that is dense on top and sparse below exercises both and the hand-over between them
+    L = configs.ConvLayer("mixed", 2, 64, 24, 24, 16, 3, 3, 1, 1, 0.05)
+    x = L.inputs(stream=31)
+    x[:, :, :12, :] = dab_synth.dense_activations((2, 64, 12, 24), stream=32)
+    x[1, :, 12:, :12] = 0.0                                      # and a block of constant (all-zero) patches
+    _check_conv(dab, x, L.weights(stream=31), 3, 3, (1, 1), (1, 1))
+
+
 def test_conv_host_entry_point(dab):
     L = configs.ConvLayer("t", 2, 16, 12, 12, 24, 3, 3, 1, 1)
     x, w = L.inputs(stream=5), L.weights(stream=5)
