@@ -108,6 +108,22 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Slowest rank's time (the job is as slow as its slowest replica)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_rank_step: float, steps: int, seconds: float, world: int) -> float:
+    """Whole-job throughput of `world` independent replicas, each doing `steps` steps in `seconds` (max over ranks)."""
+    return world * units_per_rank_step * steps / seconds
+
+
 def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
@@ -272,14 +288,10 @@ def run_dab(args):
     barrier()
     clocks = sampler.stop()
     total_ms = t_start.elapsed_time(t_end)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
 
     ops_per_step = sum(L.binary_ops for L in layers)
-    value = world * ops_per_step * args.steps / (total_ms * 1e-3) / 1e12
+    value = aggregate_throughput(ops_per_step, args.steps, total_ms * 1e-3, world) / 1e12
 
     # per-kernel device time inside the timed region
     k_ms = {"binarize_rows": 0.0, "binarize_patches": 0.0, "contract": 0.0}
@@ -343,12 +355,8 @@ def run_dab(args):
             e2e_step()
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
-        e2e = {"value": world * ops_per_step * args.e2e_steps / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e_s = max_over_ranks(e2e_s, world, dev)
+        e2e = {"value": aggregate_throughput(ops_per_step, args.e2e_steps, e2e_s, world) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * e2e_s / args.e2e_steps}
 
     cpu_baseline = None
