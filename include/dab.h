@@ -150,10 +150,14 @@ dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d
                                     const float* d_wbeta, float* d_y, int32_t* d_p11, void* stream);
 
 /*
- * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory: copies h_x
- * to the device, runs dab_binary_conv, copies the result to h_y, all on `stream`, and returns after
- * the stream has drained.  Pinned host memory makes the copies asynchronous to other streams.
- * The scratch must hold dab_binary_conv_host_workspace(desc) bytes (input + output + conv scratch).
+ * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up
+ * to 8 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
+ * chunks overlap on three streams, and the call returns after everything has drained.  Use pinned host memory:
+ * with pageable memory the copies are staged by the driver and do not overlap.  The two copy streams and a few
+ * events are created on the first call on a device and kept for the life of the process (the only state the
+ * library keeps besides dab_binary_conv_static's array); calls on one device are serialised by a lock.
+ * The scratch must hold dab_binary_conv_host_workspace(desc) bytes (two input and two output chunk buffers plus
+ * the conv scratch of one chunk).
  */
 size_t dab_binary_conv_host_workspace(const dab_conv_desc* desc);
 dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,

@@ -1,4 +1,7 @@
-// C ABI of libdab: argument validation on the host, then launches.  No allocation, no global state.
+// C ABI of libdab: argument validation on the host, then launches.  No device memory is allocated; the only
+// state kept is the pair of copy streams of the host-buffer convolution.
+#include <mutex>
+
 #include "common.cuh"
 
 using namespace dab;
@@ -186,37 +189,127 @@ dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const ui
   return dab_binary_conv_contract(desc, pm, ldm, pK, pg, pd, d_wmask, ldw, d_wK, d_walpha, d_wbeta, d_y, d_p11, stream);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Host-buffer convolution: the batch is cut into chunks of images and pipelined over three streams
+// (copy-in | compute | copy-out) with two device buffers per direction, so that PCIe traffic in both directions
+// overlaps the kernels.  The two copy streams and the events are created once per device and kept.
+// ---------------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kHostChunks = 8;  // chunks per call at most
+
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, in_done[2] = {}, comp_done[2] = {}, out_done[2] = {};
+};
+
+std::mutex g_host_mutex;
+HostPipe g_host_pipe[64];
+
+cudaError_t host_pipe(HostPipe** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  HostPipe& p = g_host_pipe[dev];
+  if (!p.ready) {
+    if ((e = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming)) != cudaSuccess) return e;
+    for (int b = 0; b < 2; ++b) {
+      if ((e = cudaEventCreateWithFlags(&p.in_done[b], cudaEventDisableTiming)) != cudaSuccess) return e;
+      if ((e = cudaEventCreateWithFlags(&p.comp_done[b], cudaEventDisableTiming)) != cudaSuccess) return e;
+      if ((e = cudaEventCreateWithFlags(&p.out_done[b], cudaEventDisableTiming)) != cudaSuccess) return e;
+    }
+    p.ready = true;
+  }
+  *out = &p;
+  return cudaSuccess;
+}
+
+struct HostPlan {
+  int32_t chunk_imgs, chunks;
+  size_t x_chunk, y_chunk, scratch, total;  // bytes (x_chunk, y_chunk rounded up to kAlign)
+  size_t x_img, y_img;                      // bytes per image
+};
+
+bool host_plan(const dab_conv_desc* desc, const ConvGeom& g, HostPlan* p) {
+  p->chunk_imgs = (desc->N + kHostChunks - 1) / kHostChunks;
+  p->chunks = (desc->N + p->chunk_imgs - 1) / p->chunk_imgs;
+  p->x_img = (size_t)desc->C * desc->H * desc->W * sizeof(float);
+  p->y_img = (size_t)desc->Cout * g.Ho * g.Wo * sizeof(float);
+  p->x_chunk = round_up(p->x_img * p->chunk_imgs, kAlign);
+  p->y_chunk = round_up(p->y_img * p->chunk_imgs, kAlign);
+  dab_conv_desc d = *desc;
+  d.N = p->chunk_imgs;
+  ConvGeom gc;
+  if (!conv_geom(&d, &gc)) return false;
+  p->scratch = conv_scratch(gc).total;
+  p->total = 2 * p->x_chunk + 2 * p->y_chunk + p->scratch;
+  return true;
+}
+
+}  // namespace
+
 size_t dab_binary_conv_host_workspace(const dab_conv_desc* desc) {
   ConvGeom g;
-  if (!conv_geom(desc, &g)) return 0;
-  size_t xb = round_up((size_t)desc->N * desc->C * desc->H * desc->W * sizeof(float), kAlign);
-  size_t yb = round_up((size_t)g.patches * desc->Cout * sizeof(float), kAlign);
-  return xb + yb + conv_scratch(g).total;
+  HostPlan p;
+  if (!conv_geom(desc, &g) || !host_plan(desc, g, &p)) return 0;
+  return p.total;
 }
 
 dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,
                                 const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* h_y,
                                 void* d_workspace, size_t workspace_bytes, void* stream) {
   ConvGeom g;
-  if (!conv_geom(desc, &g)) return DAB_ERR_INVALID_ARG;
+  HostPlan pl;
+  if (!conv_geom(desc, &g) || !host_plan(desc, g, &pl)) return DAB_ERR_INVALID_ARG;
   if (!h_x || !h_y) return DAB_ERR_INVALID_ARG;
-  size_t need = dab_binary_conv_host_workspace(desc);
-  if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign) || workspace_bytes < need)
+  if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign) || workspace_bytes < pl.total)
     return DAB_ERR_WORKSPACE;
+  std::lock_guard<std::mutex> lock(g_host_mutex);  // the copy streams and events are shared by all calls
+  HostPipe* hp = nullptr;
+  if (host_pipe(&hp) != cudaSuccess) return DAB_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  size_t x_bytes = (size_t)desc->N * desc->C * desc->H * desc->W * sizeof(float);
-  size_t y_bytes = (size_t)g.patches * desc->Cout * sizeof(float);
-  size_t xb = round_up(x_bytes, kAlign), yb = round_up(y_bytes, kAlign);
   char* ws = static_cast<char*>(d_workspace);
-  float* d_x = reinterpret_cast<float*>(ws);
-  float* d_y = reinterpret_cast<float*>(ws + xb);
-  if (cudaMemcpyAsync(d_x, h_x, x_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return DAB_ERR_CUDA;
-  dab_status s = dab_binary_conv(desc, d_x, d_wmask, ldw, d_wK, d_walpha, d_wbeta, d_y, ws + xb + yb,
-                                 workspace_bytes - xb - yb, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr,
-                                 stream);
-  if (s != DAB_OK) return s;
-  if (cudaMemcpyAsync(h_y, d_y, y_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DAB_ERR_CUDA;
-  return from_cuda(cudaStreamSynchronize(st));
+  float* xbuf[2] = {reinterpret_cast<float*>(ws), reinterpret_cast<float*>(ws + pl.x_chunk)};
+  float* ybuf[2] = {reinterpret_cast<float*>(ws + 2 * pl.x_chunk), reinterpret_cast<float*>(ws + 2 * pl.x_chunk + pl.y_chunk)};
+  char* scratch = ws + 2 * pl.x_chunk + 2 * pl.y_chunk;
+
+#define DAB_TRY(call) do { if ((call) != cudaSuccess) { cudaStreamSynchronize(hp->in); cudaStreamSynchronize(hp->out); \
+                           cudaStreamSynchronize(st); return DAB_ERR_CUDA; } } while (0)
+  DAB_TRY(cudaEventRecord(hp->start, st));  // work already queued on the caller's stream comes first
+  DAB_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+  dab_status status = DAB_OK;
+  for (int c = 0; c < pl.chunks; ++c) {
+    const int b = c & 1;
+    const int32_t img0 = c * pl.chunk_imgs;
+    const int32_t imgs = desc->N - img0 < pl.chunk_imgs ? desc->N - img0 : pl.chunk_imgs;
+    // copy-in: the x buffer is free once the chunk that used it two rounds ago has been computed
+    if (c >= 2) DAB_TRY(cudaStreamWaitEvent(hp->in, hp->comp_done[b], 0));
+    DAB_TRY(cudaMemcpyAsync(xbuf[b], reinterpret_cast<const char*>(h_x) + (size_t)img0 * pl.x_img, pl.x_img * imgs,
+                            cudaMemcpyHostToDevice, hp->in));
+    DAB_TRY(cudaEventRecord(hp->in_done[b], hp->in));
+    // compute: needs the input, and the y buffer must have been copied out
+    DAB_TRY(cudaStreamWaitEvent(st, hp->in_done[b], 0));
+    if (c >= 2) DAB_TRY(cudaStreamWaitEvent(st, hp->out_done[b], 0));
+    dab_conv_desc d = *desc;
+    d.N = imgs;
+    status = dab_binary_conv(&d, xbuf[b], d_wmask, ldw, d_wK, d_walpha, d_wbeta, ybuf[b], scratch, pl.scratch, nullptr,
+                             nullptr, nullptr, nullptr, 0, nullptr, nullptr, stream);
+    if (status != DAB_OK) break;
+    DAB_TRY(cudaEventRecord(hp->comp_done[b], st));
+    // copy-out
+    DAB_TRY(cudaStreamWaitEvent(hp->out, hp->comp_done[b], 0));
+    DAB_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(h_y) + (size_t)img0 * pl.y_img, ybuf[b], pl.y_img * imgs,
+                            cudaMemcpyDeviceToHost, hp->out));
+    DAB_TRY(cudaEventRecord(hp->out_done[b], hp->out));
+  }
+#undef DAB_TRY
+  cudaError_t e1 = cudaStreamSynchronize(hp->in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(hp->out);
+  if (status != DAB_OK) return status;
+  return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess) ? DAB_OK : DAB_ERR_CUDA;
 }
 
 dab_status dab_popc_probe(uint32_t* d_sink, int32_t blocks, int32_t iters, void* stream) {

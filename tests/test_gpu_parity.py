@@ -215,13 +215,19 @@ def test_conv_with_dense_and_sparse_regions(dab):
     _check_conv(dab, x, L.weights(stream=31), 3, 3, (1, 1), (1, 1))
 
 
-def test_conv_host_entry_point(dab):
-    L = configs.ConvLayer("t", 2, 16, 12, 12, 24, 3, 3, 1, 1)
+@pytest.mark.parametrize("batch", [1, 2, 19])
+def test_conv_host_entry_point(dab, batch):
+    # host tensors in and out; the batch is pipelined in chunks (19 images: 7 chunks, the last one ragged)
+    L = configs.ConvLayer("t", batch, 16, 12, 12, 24, 3, 3, 1, 1)
     x, w = L.inputs(stream=5), L.weights(stream=5)
     wd = dab.dab_binarize(to_dev(w))
     y_dev = dab.dab_binary_conv(to_dev(x), wd, 3, 3, (1, 1), (1, 1)).cpu()
-    y_host = dab.dab_binary_conv_host(torch.from_numpy(x).pin_memory(), wd, 3, 3, (1, 1), (1, 1))
-    assert torch.equal(y_host, y_dev)
+    for _ in range(2):                                           # twice: the copy streams and events are reused
+        y_host = dab.dab_binary_conv_host(torch.from_numpy(x).pin_memory(), wd, 3, 3, (1, 1), (1, 1))
+        assert torch.equal(y_host, y_dev)
+    y_pageable = dab.dab_binary_conv_host(torch.from_numpy(x), wd, 3, 3, (1, 1), (1, 1),
+                                          y_host=torch.empty_like(y_dev))
+    assert torch.equal(y_pageable, y_dev)
 
 
 def test_argument_errors_are_return_codes(dab):
