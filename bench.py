@@ -29,6 +29,15 @@ WORDS_PER_POPC = 1.5              # the contraction compresses 3 AND-ed words in
 SM_COUNT = 148
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the patch-coder launches of each layer at batch 256, from one
+# ncu capture of this benchmark (profiles/binarize_patches_dram_traffic_config5.md).  Valid for the kernels as
+# they were then: reset to {} when the patch coder changes.
+PATCH_CODER_DRAM_BYTES = {"l1_0": 274342912, "l1_1": 270581760, "l1_2": 272141056, "l1_3": 271047936, "l2_0": 221521408,
+                          "l2_1": 120040960, "l2_2": 119217920, "l2_3": 119235584, "l3_0": 107264000, "l3_1": 52955136,
+                          "l3_2": 53775104, "l3_3": 53685760, "l4_0": 52193280, "l4_1": 26870272, "l4_2": 26882304,
+                          "l4_3": 26891008}
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -305,8 +314,13 @@ def run_dab(args):
     # (4*ceil(n/32) B) and K, gamma, delta (12 B) written
     patch_bytes = sum(4 * L.N * L.C * L.H * L.W + L.patches * (4 * dab.dab_words_per_row(L.n) + 12) for L in layers)
     binarize_gbs = patch_bytes * args.steps / (k_ms["binarize_patches"] * 1e-3) / 1e9
-    roofline = {"kernel": "binarize_patches_kernel", "bound": "hbm", "achieved": binarize_gbs, "peak": hbm_peak,
-                "unit": "GB/s", "frac": binarize_gbs / hbm_peak, "traffic": None, "peak_source": peak_src,
+    traffic = None
+    if args.batch == 256 and not args.dense and all(L.name in PATCH_CODER_DRAM_BYTES for L in layers):
+        traffic = sum(PATCH_CODER_DRAM_BYTES[L.name] for L in layers) / len(layers)   # per layer launch, like achieved
+    roofline = {"kernel": "binarize_patches_{warp,group}_kernel", "bound": "hbm", "achieved": binarize_gbs,
+                "peak": hbm_peak, "unit": "GB/s", "frac": binarize_gbs / hbm_peak, "traffic": traffic,
+                "traffic_note": "measured DRAM bytes per layer launch (ncu), average over the layers; algorithmic "
+                                "average alongside", "peak_source": peak_src,
                 "algorithmic_bytes_per_launch_avg": patch_bytes / len(layers),
                 "avg_launch_ms": k_ms["binarize_patches"] / launches_per_kind,
                 "share_of_step": k_ms["binarize_patches"] / sum(k_ms.values())}
