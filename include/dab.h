@@ -150,6 +150,28 @@ dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d
                                     const float* d_wbeta, float* d_y, int32_t* d_p11, void* stream);
 
 /*
+ * Sign coding — the input coding of the paper's fully binarized ("FBin") layers, which are "structured the same
+ * as the XNOR-Net" (Appendix, "Experimental details"): mask bit = [x >= 0], gamma = mean |x| over the row,
+ * delta = -gamma.  It is the special case alpha = -beta of Section 4.1 (no search, no sort).  Outputs have the
+ * layout of dab_binarize / dab_binarize_patches, so the contraction calls take them unchanged.  -0.0 counts as
+ * +0.0; rows with a NaN or an infinity get DAB_ROW_NONFINITE, K = 0, an empty mask and NaN scales.
+ *
+ * dab_sign_binarize        rows of a matrix (arguments as dab_binarize)
+ * dab_sign_patches         patches of an NCHW tensor (arguments as dab_binarize_patches)
+ * dab_binary_conv_sign     dab_sign_patches + dab_binary_conv_contract (arguments as dab_binary_conv)
+ */
+dab_status dab_sign_binarize(const float* d_values, int64_t rows, int32_t n, int64_t ld_values, int32_t* d_K,
+                             float* d_alpha, float* d_beta, uint32_t* d_mask, int32_t ld_mask, uint32_t* d_row_flags,
+                             void* stream);
+dab_status dab_sign_patches(const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
+                            float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream);
+dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                                const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
+                                void* d_workspace, size_t workspace_bytes, int32_t* d_pK, float* d_pgamma,
+                                float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, int32_t* d_p11,
+                                void* stream);
+
+/*
  * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up
  * to 8 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
  * chunks overlap on three streams, and the call returns after everything has drained.  Use pinned host memory:

@@ -86,6 +86,19 @@ def binarize(values: np.ndarray) -> Binarized:
     return out
 
 
+def sign_code(values: np.ndarray) -> Binarized:
+    """Rows -> sign masks with one scale (alpha = mean|w|, beta = -alpha): the XNOR-style code of FBin inputs."""
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    rows, n = v.shape
+    out = Binarized(np.zeros((rows, n), np.uint8), np.zeros(rows, np.int32), np.zeros(rows, np.float32),
+                    np.zeros(rows, np.float32), np.zeros(rows, np.uint32), np.zeros(rows, np.int32),
+                    np.zeros(rows, np.float64), np.full(rows, np.inf))
+    if rows and n:
+        lib().oracle_sign(_p(v), C.c_int64(rows), C.c_int32(n), C.c_int64(n), _p(out.e), _p(out.K), _p(out.alpha),
+                          _p(out.beta), _p(out.flags))
+    return out
+
+
 def pack(bits: np.ndarray, ld_mask: int | None = None):
     """0/1 bytes (rows x n) -> (uint32 words rows x ld_mask, K per row)."""
     b = np.ascontiguousarray(bits, dtype=np.uint8)
@@ -136,8 +149,9 @@ def _desc(x_shape, Cout, kh, kw, stride, pad):
     return ConvDesc(N, Cc, H, W, Cout, kh, kw, stride[0], stride[1], pad[0], pad[1])
 
 
-def conv(x, w_e, w_alpha, w_beta, kh, kw, stride=(1, 1), pad=(0, 0), details=True) -> ConvResult:
-    """Binary forward pass I (*) W~ (Section 4.3.2), every patch coded by Algorithm 1."""
+def conv(x, w_e, w_alpha, w_beta, kh, kw, stride=(1, 1), pad=(0, 0), details=True, sign_inputs=False) -> ConvResult:
+    """Binary forward pass I (*) W~ (Section 4.3.2), every patch coded by Algorithm 1 (sign_inputs: by its sign
+    pattern and mean magnitude instead, as in the paper's XNOR-structured FBin layers)."""
     x = np.ascontiguousarray(x, np.float32)
     w_e = np.ascontiguousarray(w_e, np.uint8)
     w_alpha = np.ascontiguousarray(w_alpha, np.float32)
@@ -155,7 +169,8 @@ def conv(x, w_e, w_alpha, w_beta, kh, kw, stride=(1, 1), pad=(0, 0), details=Tru
         p_f, p_p = np.zeros(P, np.uint32), np.zeros((P, Cout), np.int32)
     else:
         p_e = p_K = p_g = p_d = p_f = p_p = None
-    lib().oracle_conv(C.byref(d), _p(x), _p(w_e), _p(w_alpha), _p(w_beta), _p(y), _p(p_e), _p(p_K), _p(p_g), _p(p_d),
+    fn = lib().oracle_conv_sign if sign_inputs else lib().oracle_conv
+    fn(C.byref(d), _p(x), _p(w_e), _p(w_alpha), _p(w_beta), _p(y), _p(p_e), _p(p_K), _p(p_g), _p(p_d),
                       _p(p_f), _p(p_p))
     return ConvResult(y, p_e, p_K, p_g, p_d, p_f, p_p)
 

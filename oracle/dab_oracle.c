@@ -129,6 +129,35 @@ void oracle_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_va
   }
 }
 
+void oracle_sign_row(const float* w, int32_t n, uint8_t* e, int32_t* K, float* alpha, float* beta, uint32_t* flags) {
+  int32_t i, k = 0;
+  double sum = 0.0;
+  memset(e, 0, (size_t)n);
+  *K = 0;
+  *flags = 0;
+  for (i = 0; i < n; ++i)
+    if (!isfinite(w[i])) *flags |= ORACLE_FLAG_NONFINITE;
+  if (*flags) {
+    *alpha = *beta = NAN;
+    return;
+  }
+  for (i = 0; i < n; ++i) {
+    sum += fabs((double)w[i]);
+    e[i] = (uint8_t)((double)w[i] >= 0.0);
+    k += e[i];
+  }
+  *K = k;
+  *alpha = (float)(sum / (double)n);
+  *beta = -*alpha;
+}
+
+void oracle_sign(const float* values, int64_t rows, int32_t n, int64_t ld_values, uint8_t* e, int32_t* K, float* alpha,
+                 float* beta, uint32_t* flags) {
+  int64_t r;
+  for (r = 0; r < rows; ++r)
+    oracle_sign_row(values + r * ld_values, n, e + r * (int64_t)n, K + r, alpha + r, beta + r, flags + r);
+}
+
 void oracle_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld_bits, uint32_t* mask, int32_t ld_mask,
                  int32_t* K) {
   int64_t r;
@@ -209,9 +238,9 @@ void oracle_im2col(const oracle_conv_desc* d, const float* x, float* patches) {
         extract_patch(d, x, img, ho, wo, patches + (((int64_t)img * Ho + ho) * Wo + wo) * n);
 }
 
-void oracle_conv(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
-                 const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K, float* p_gamma, float* p_delta,
-                 uint32_t* p_flags, int32_t* p_p11) {
+static void conv_with_coder(int sign_coder, const oracle_conv_desc* d, const float* x, const uint8_t* w_e,
+                            const float* w_alpha, const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K,
+                            float* p_gamma, float* p_delta, uint32_t* p_flags, int32_t* p_p11) {
   int32_t Ho, Wo;
   int32_t n = d->C * d->kh * d->kw;
   int64_t patches, pi;
@@ -230,7 +259,8 @@ void oracle_conv(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, 
     float gamma, delta;
     uint32_t fl;
     extract_patch(d, x, img, ho, wo, p);
-    oracle_binarize_row(p, n, f, &Kf, &gamma, &delta, &fl, 0, 0, 0);
+    if (sign_coder) oracle_sign_row(p, n, f, &Kf, &gamma, &delta, &fl);
+    else oracle_binarize_row(p, n, f, &Kf, &gamma, &delta, &fl, 0, 0, 0);
     if (p_e) memcpy(p_e + pi * (int64_t)n, f, (size_t)n);
     if (p_K) p_K[pi] = Kf;
     if (p_gamma) p_gamma[pi] = gamma;
@@ -245,4 +275,16 @@ void oracle_conv(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, 
     free(p);
     free(f);
   }
+}
+
+void oracle_conv(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
+                 const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K, float* p_gamma, float* p_delta,
+                 uint32_t* p_flags, int32_t* p_p11) {
+  conv_with_coder(0, d, x, w_e, w_alpha, w_beta, y, p_e, p_K, p_gamma, p_delta, p_flags, p_p11);
+}
+
+void oracle_conv_sign(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
+                      const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K, float* p_gamma, float* p_delta,
+                      uint32_t* p_flags, int32_t* p_p11) {
+  conv_with_coder(1, d, x, w_e, w_alpha, w_beta, y, p_e, p_K, p_gamma, p_delta, p_flags, p_p11);
 }

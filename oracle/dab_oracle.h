@@ -47,6 +47,16 @@ void oracle_binarize_row(const float* w, int32_t n, uint8_t* e, int32_t* K, floa
 void oracle_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_values, uint8_t* e, int32_t* K,
                      float* alpha, float* beta, uint32_t* flags, int32_t* s_star, double* best_D, double* gap);
 
+/*
+ * Sign coding with one scale (the XNOR-Net code the paper's fully binarized layers use for their inputs,
+ * Appendix "Experimental details"; the special case alpha = -beta of Section 4.1):
+ *   e_i = [w_i >= 0], alpha = mean |w_i|, beta = -alpha, K = number of ones.  -0.0 counts as +0.0.
+ * flags: ORACLE_FLAG_NONFINITE as above (then alpha = beta = NaN, empty mask); no row is degenerate here.
+ */
+void oracle_sign_row(const float* w, int32_t n, uint8_t* e, int32_t* K, float* alpha, float* beta, uint32_t* flags);
+void oracle_sign(const float* values, int64_t rows, int32_t n, int64_t ld_values, uint8_t* e, int32_t* K, float* alpha,
+                 float* beta, uint32_t* flags);
+
 /* Bit packing: bit (i mod 32) of word (i div 32) of a row is e_i; words up to ld_mask and bits beyond n are 0.
  * K (nullable) receives the number of ones per row. */
 void oracle_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld_bits, uint32_t* mask, int32_t ld_mask,
@@ -79,6 +89,11 @@ typedef struct {
 void oracle_conv(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
                  const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K, float* p_gamma, float* p_delta,
                  uint32_t* p_flags, int32_t* p_p11);
+
+/* The same forward pass with every input patch coded by oracle_sign_row instead (paper-faithful FBin inputs). */
+void oracle_conv_sign(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
+                      const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K, float* p_gamma, float* p_delta,
+                      uint32_t* p_flags, int32_t* p_p11);
 
 /* Patch extraction alone (explicit loops), rows = N*Ho*Wo, row length C*kh*kw. */
 void oracle_im2col(const oracle_conv_desc* d, const float* x, float* patches);

@@ -22,7 +22,7 @@ ROW_NONFINITE = 2
 
 EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_binarize", "dab_pack", "dab_binary_gemm",
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
-           "dab_binary_conv_contract", "dab_binary_conv_host_workspace",
+           "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe")
 
 
@@ -61,6 +61,9 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_host_workspace.argtypes = [vp]
         L.dab_binary_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp, vp, vp, vp, i32, vp, vp, vp]
         L.dab_binarize_patches.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp]
+        L.dab_sign_patches.argtypes = L.dab_binarize_patches.argtypes
+        L.dab_sign_binarize.argtypes = L.dab_binarize.argtypes
+        L.dab_binary_conv_sign.argtypes = L.dab_binary_conv.argtypes
         L.dab_binary_conv_contract.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.dab_binary_conv_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.dab_binary_conv_static_capacity.restype = C.c_size_t
@@ -118,7 +121,12 @@ class Coded:
         return self.mask.shape[1]
 
 
-def dab_binarize(values: torch.Tensor, ld_mask: int | None = None, stream=None) -> Coded:
+def dab_sign_binarize(values: torch.Tensor, ld_mask: int | None = None, stream=None) -> "Coded":
+    """Sign coding of rows (mask = [x >= 0], alpha = mean|x|, beta = -alpha); outputs as dab_binarize."""
+    return dab_binarize(values, ld_mask, stream, _entry="dab_sign_binarize")
+
+
+def dab_binarize(values: torch.Tensor, ld_mask: int | None = None, stream=None, _entry: str = "dab_binarize") -> Coded:
     """rows x n fp32 (row stride = values.stride(0)) -> K, alpha, beta, packed mask, flags."""
     _dev(values, torch.float32, "values")
     if values.dim() != 2 or values.stride(1) != 1:
@@ -130,9 +138,9 @@ def dab_binarize(values: torch.Tensor, ld_mask: int | None = None, stream=None) 
                 torch.empty(rows, dtype=torch.float32, device=dev), torch.empty(rows, dtype=torch.float32, device=dev),
                 torch.empty(rows, dtype=torch.int32, device=dev), n)
     ldv = values.stride(0) if rows > 1 else max(n, values.stride(0))
-    st = lib().dab_binarize(_ptr(values), rows, n, ldv, _ptr(out.K), _ptr(out.alpha), _ptr(out.beta), _ptr(out.mask),
-                            ld, _ptr(out.flags), _stream(stream))
-    _check(st, "dab_binarize")
+    st = getattr(lib(), _entry)(_ptr(values), rows, n, ldv, _ptr(out.K), _ptr(out.alpha), _ptr(out.beta),
+                                _ptr(out.mask), ld, _ptr(out.flags), _stream(stream))
+    _check(st, _entry)
     return out
 
 
@@ -204,8 +212,10 @@ class ConvDetails:
 
 
 def dab_binary_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0), details: bool = False,
-                    y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None):
-    """x: N x C x H x W fp32 (contiguous); w: filters coded by dab_binarize on [Cout x C*kh*kw] -> y NCHW fp32."""
+                    y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None,
+                    sign_inputs: bool = False):
+    """x: N x C x H x W fp32 (contiguous); w: filters coded by dab_binarize on [Cout x C*kh*kw] -> y NCHW fp32.
+    sign_inputs: code the patches by sign and mean magnitude (dab_binary_conv_sign) instead of the optimal split."""
     _dev(x, torch.float32, "x")
     if not x.is_contiguous():
         raise ValueError("x must be contiguous NCHW")
@@ -228,7 +238,8 @@ def dab_binary_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), 
                           torch.empty((P, dab_default_ld(w.n)), dtype=torch.int32, device=dev),
                           torch.empty(P, dtype=torch.int32, device=dev),
                           torch.empty((P, Cout), dtype=torch.int32, device=dev))
-    st = lib().dab_binary_conv(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha), _ptr(w.beta),
+    entry = lib().dab_binary_conv_sign if sign_inputs else lib().dab_binary_conv
+    st = entry(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha), _ptr(w.beta),
                                _ptr(y), _ptr(workspace), workspace.numel(),
                                _ptr(det.pK) if det else None, _ptr(det.pgamma) if det else None,
                                _ptr(det.pdelta) if det else None, _ptr(det.pmask) if det else None,
@@ -236,6 +247,13 @@ def dab_binary_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), 
                                _ptr(det.p11) if det else None, _stream(stream))
     _check(st, "dab_binary_conv")
     return (y, det) if details else y
+
+
+def dab_sign_patches(desc: ConvDesc, x: torch.Tensor, pK, pgamma, pdelta, pmask, pflags=None, stream=None) -> None:
+    """Sign coding of every patch (stage 1 of dab_binary_conv_sign) with caller-provided outputs."""
+    st = lib().dab_sign_patches(C.byref(desc), _ptr(x), _ptr(pK), _ptr(pgamma), _ptr(pdelta), _ptr(pmask),
+                                pmask.stride(0), _ptr(pflags), _stream(stream))
+    _check(st, "dab_sign_patches")
 
 
 def dab_binarize_patches(desc: ConvDesc, x: torch.Tensor, pK, pgamma, pdelta, pmask, pflags=None, stream=None) -> None:

@@ -127,8 +127,8 @@ size_t dab_binary_conv_workspace(const dab_conv_desc* desc) {
   return conv_scratch(g).total;
 }
 
-dab_status dab_binarize_patches(const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
-                                float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream) {
+static dab_status code_patches(bool sign, const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
+                               float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream) {
   if (!desc) return DAB_ERR_INVALID_ARG;
   if (desc->C > 0 && desc->kh > 0 && desc->kw > 0 && (int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N)
     return DAB_ERR_UNSUPPORTED;
@@ -136,8 +136,32 @@ dab_status dab_binarize_patches(const dab_conv_desc* desc, const float* d_x, int
   if (!conv_geom(desc, &g)) return DAB_ERR_INVALID_ARG;
   if (!d_x || !d_pK || !d_pgamma || !d_pdelta || !d_pmask) return DAB_ERR_INVALID_ARG;
   if (ldp < dab_words_per_row(g.n) || (ldp & 3) || !aligned16(d_pmask)) return DAB_ERR_INVALID_ARG;
-  return from_cuda(launch_binarize_patches(*desc, g.Ho, g.Wo, d_x, d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags,
-                                           static_cast<cudaStream_t>(stream)));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return from_cuda(sign ? launch_sign_patches(*desc, g.Ho, g.Wo, d_x, d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags, st)
+                        : launch_binarize_patches(*desc, g.Ho, g.Wo, d_x, d_pK, d_pgamma, d_pdelta, d_pmask, ldp,
+                                                  d_pflags, st));
+}
+
+dab_status dab_binarize_patches(const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
+                                float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream) {
+  return code_patches(false, desc, d_x, d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags, stream);
+}
+
+dab_status dab_sign_patches(const dab_conv_desc* desc, const float* d_x, int32_t* d_pK, float* d_pgamma,
+                            float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, void* stream) {
+  return code_patches(true, desc, d_x, d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags, stream);
+}
+
+dab_status dab_sign_binarize(const float* d_values, int64_t rows, int32_t n, int64_t ld_values, int32_t* d_K,
+                             float* d_alpha, float* d_beta, uint32_t* d_mask, int32_t ld_mask, uint32_t* d_row_flags,
+                             void* stream) {
+  if (rows < 0 || n < 1) return DAB_ERR_INVALID_ARG;
+  if (n > DAB_MAX_N) return DAB_ERR_UNSUPPORTED;
+  if (ld_values < n || ld_mask < dab_words_per_row(n) || (ld_mask & 3)) return DAB_ERR_INVALID_ARG;
+  if (rows == 0) return DAB_OK;
+  if (!d_values || !d_K || !d_alpha || !d_beta || !d_mask || !aligned16(d_mask)) return DAB_ERR_INVALID_ARG;
+  return from_cuda(launch_sign_rows(d_values, rows, n, ld_values, d_K, d_alpha, d_beta, d_mask, ld_mask, d_row_flags,
+                                    static_cast<cudaStream_t>(stream)));
 }
 
 dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d_pmask, int32_t ldp,
@@ -163,7 +187,7 @@ dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d
   return from_cuda(launch_gemm(a, /*lanes_along_rows=*/true, static_cast<cudaStream_t>(stream)));
 }
 
-dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+static dab_status conv_with_coder(bool sign, const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
                            const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
                            void* d_workspace, size_t workspace_bytes, int32_t* d_pK, float* d_pgamma,
                            float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, int32_t* d_p11,
@@ -184,9 +208,27 @@ dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const ui
   float* pd = d_pdelta ? d_pdelta : reinterpret_cast<float*>(ws + sc.off_delta);
   uint32_t* pm = d_pmask ? d_pmask : reinterpret_cast<uint32_t*>(ws + sc.off_mask);
   int32_t ldm = d_pmask ? ldp : g.ld;
-  dab_status s = dab_binarize_patches(desc, d_x, pK, pg, pd, pm, ldm, d_pflags, stream);
+  dab_status s = code_patches(sign, desc, d_x, pK, pg, pd, pm, ldm, d_pflags, stream);
   if (s != DAB_OK) return s;
   return dab_binary_conv_contract(desc, pm, ldm, pK, pg, pd, d_wmask, ldw, d_wK, d_walpha, d_wbeta, d_y, d_p11, stream);
+}
+
+dab_status dab_binary_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                           const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
+                           void* d_workspace, size_t workspace_bytes, int32_t* d_pK, float* d_pgamma,
+                           float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, int32_t* d_p11,
+                           void* stream) {
+  return conv_with_coder(false, desc, d_x, d_wmask, ldw, d_wK, d_walpha, d_wbeta, d_y, d_workspace, workspace_bytes,
+                         d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags, d_p11, stream);
+}
+
+dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                                const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
+                                void* d_workspace, size_t workspace_bytes, int32_t* d_pK, float* d_pgamma,
+                                float* d_pdelta, uint32_t* d_pmask, int32_t ldp, uint32_t* d_pflags, int32_t* d_p11,
+                                void* stream) {
+  return conv_with_coder(true, desc, d_x, d_wmask, ldw, d_wK, d_walpha, d_wbeta, d_y, d_workspace, workspace_bytes,
+                         d_pK, d_pgamma, d_pdelta, d_pmask, ldp, d_pflags, d_p11, stream);
 }
 
 // ---------------------------------------------------------------------------------------------------------

@@ -73,6 +73,11 @@ cudaError_t launch_gemm(const GemmArgs& args, bool lanes_along_rows, cudaStream_
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
                                     float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
                                     cudaStream_t stream);
+cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K, float* alpha,
+                             float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags, cudaStream_t stream);
+cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
+                                float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
+                                cudaStream_t stream);
 cudaError_t launch_popc_probe(uint32_t* sink, int32_t blocks, int32_t iters, cudaStream_t stream);
 
 }  // namespace dab

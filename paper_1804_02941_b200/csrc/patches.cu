@@ -195,6 +195,98 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Sign coding (the paper's XNOR-structured FBin inputs): mask bit = [x >= 0], gamma = mean |x|, delta = -gamma.
+// One warp per row; `value(i)` returns element i.  HBM-bound work: no sort, one pass.
+// ---------------------------------------------------------------------------------------------------------
+template <typename Value>
+__device__ __forceinline__ void warp_sign_row(Value value, int n, int ld, int lane, int32_t* K_out, float* gamma_out,
+                                              float* delta_out, uint32_t* flags_out, uint32_t* __restrict__ mrow) {
+  double sum = 0.0;
+  int ones = 0, bad = 0;
+  uint32_t mine = 0;
+  const int words = (n + 31) >> 5;
+  for (int k = 0; k < words; ++k) {
+    const int i = k * 32 + lane;
+    float x = -1.0f;  // lanes beyond n contribute a 0 bit
+    if (i < n) {
+      x = value(i);
+      bad |= is_nonfinite(x);
+      sum += fabs((double)x);
+    }
+    const uint32_t word = __ballot_sync(0xFFFFFFFFu, i < n && x >= 0.0f);
+    ones += __popc(word);
+    if ((k & 31) == lane) mine = word;
+    if ((k & 31) == 31 || k == words - 1) {  // a batch of up to 32 words is complete: one coalesced store
+      const int w = (k & ~31) + lane;
+      if (w <= k) mrow[w] = mine;
+    }
+  }
+  for (int w = words + lane; w < ld; w += 32) mrow[w] = 0u;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, off);
+  bad = __any_sync(0xFFFFFFFFu, bad);
+  if (bad) {  // flagged rows: empty mask, NaN scales
+    __syncwarp();
+    for (int w = lane; w < ld; w += 32) mrow[w] = 0u;
+  }
+  if (lane == 0) {
+    const float g = bad ? __uint_as_float(0x7FC00000u) : (float)(sum / (double)n);
+    *K_out = bad ? 0 : ones;
+    *gamma_out = g;
+    *delta_out = -g;
+    if (flags_out) *flags_out = bad ? DAB_ROW_NONFINITE : 0u;
+  }
+}
+
+__global__ void __launch_bounds__(kWarpsPerCta * 32) sign_patches_kernel(const PatchArgs a) {
+  constexpr int THREADS = kWarpsPerCta * 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* tile = reinterpret_cast<float*>(smem_raw);
+  const int ch_words = a.in_h * a.pitch;
+  uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  fill_offsets(a, off, ch_words, threadIdx.x, THREADS);
+  const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+    const TileCoord t = tile_coord(a, tile_id);
+    __syncthreads();
+    load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
+    __syncthreads();
+    for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
+      const int lh = p / t.tw, lw = p % t.tw;
+      const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+      auto value = [origin, off](int i) { return origin[off[i]]; };
+      const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
+      warp_sign_row(value, a.n, a.ldp, lane, a.pK + pi, a.pgamma + pi, a.pdelta + pi,
+                    a.pflags ? a.pflags + pi : nullptr, a.pmask + pi * (int64_t)a.ldp);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) sign_rows_kernel(const float* __restrict__ values, int64_t rows, int32_t n,
+                                                        int64_t ld_values, int32_t* K, float* alpha, float* beta,
+                                                        uint32_t* mask, int32_t ld_mask, uint32_t* flags) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t row = warp0; row < rows; row += nwarps) {
+    const float* v = values + row * ld_values;
+    auto value = [v](int i) { return __ldg(v + i); };
+    warp_sign_row(value, n, ld_mask, lane, K + row, alpha + row, beta + row, flags ? flags + row : nullptr,
+                  mask + row * (int64_t)ld_mask);
+  }
+}
+
+cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K, float* alpha,
+                             float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags, cudaStream_t stream) {
+  int64_t blocks = (rows + 7) / 8;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  sign_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask,
+                                                        flags);
+  return cudaGetLastError();
+}
+
 // Tile shapes tried, largest first.
 static const int kTileShapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
 
@@ -254,6 +346,17 @@ static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream) {
   size_t fixed = (kTable ? sizeof(double) * rcp_table_slots(a.n) : 0) + sizeof(GroupShared) * G +
                  sizeof(uint32_t) * (size_t)a.scratch_words * G;
   return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, stream);
+}
+
+cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
+                                float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
+                                cudaStream_t stream) {
+  PatchArgs a;
+  a.d = d; a.Ho = Ho; a.Wo = Wo; a.n = d.C * d.kh * d.kw;
+  a.scratch_words = 0;
+  a.defer_dense = 0; a.marked_only = 0; a.tile_shape = -1;
+  a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
+  return launch_patches(sign_patches_kernel, a, 0, kWarpsPerCta * 32, stream);
 }
 
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,

@@ -61,6 +61,7 @@ def conv_layer(cfg, L, stream, hbm, tops_peak, dense=False):
     pm = torch.empty((P, ld), dtype=torch.int32, device=dev)
     y = torch.empty((L.N, L.Cout, L.Ho, L.Wo), device=dev)
     t_w = timed(lambda: dab.dab_binarize_into(w, wd.K, wd.alpha, wd.beta, wd.mask, wd.flags))
+    t_s = timed(lambda: dab.dab_sign_patches(desc, x, pK, pg, pd, pm, None))   # FBin-style input coding, for comparison
     t_p = timed(lambda: dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, None))
     t_c = timed(lambda: dab.dab_binary_conv_contract(desc, pm, pK, pg, pd, wd, y, None))
     wd_words = dab.dab_words_per_row(L.n)
@@ -69,6 +70,7 @@ def conv_layer(cfg, L, stream, hbm, tops_peak, dense=False):
     common = dict(config=cfg, layer=L.name, n=L.n, patches=P, filters=L.Cout, inputs="dense" if dense else "relu60")
     emit(stage="binarize_filters", ms=t_w, gbs=bytes_w / t_w / 1e6, hbm_frac=bytes_w / t_w / 1e6 / hbm, **common)
     emit(stage="binarize_patches", ms=t_p, gbs=bytes_p / t_p / 1e6, hbm_frac=bytes_p / t_p / 1e6 / hbm, **common)
+    emit(stage="sign_patches", ms=t_s, gbs=bytes_p / t_s / 1e6, hbm_frac=bytes_p / t_s / 1e6 / hbm, **common)
     emit(stage="contract", ms=t_c, tops_equiv=L.binary_ops / t_c / 1e9, alu_frac=L.binary_ops / t_c / 1e9 / tops_peak,
          **common)
     emit(stage="conv_total", ms=t_p + t_c, tops_equiv=L.binary_ops / (t_p + t_c) / 1e9, **common)

@@ -215,6 +215,31 @@ def test_conv_with_dense_and_sparse_regions(dab):
     _check_conv(dab, x, L.weights(stream=31), 3, 3, (1, 1), (1, 1))
 
 
+@pytest.mark.parametrize("n", [1, 5, 31, 32, 33, 100, 576, 577, 1025, 4608, 16384])
+def test_sign_coding_of_rows_matches_checker(dab, n):
+    w = np.concatenate([_rows("normal", 9, n, 40 + n), _rows("relu", 3, n, 41 + n), _rows("ints", 3, n, 42 + n)])
+    w[2, n // 2] = np.nan
+    got = dab.dab_sign_binarize(to_dev(w))
+    check_coded(got, oracle.sign_code(w), n)
+
+
+@pytest.mark.parametrize("ci", [0, 1, 2, 4, 5, 7, 8])
+def test_conv_with_sign_coded_inputs_matches_checker(dab, ci):
+    c = CONV_CASES[ci]
+    shape = (c["N"], c["C"], c["H"], c["W"])
+    x = dab_synth.dense_activations(shape, stream=160 + ci)
+    w = dab_synth.normal((c["Cout"], c["C"] * c["kh"] * c["kw"]), 0.05, stream=180 + ci)
+    wd, wb = dab.dab_binarize(to_dev(w)), oracle.binarize(w)
+    y, det = dab.dab_binary_conv(to_dev(x), wd, c["kh"], c["kw"], c["stride"], c["pad"], details=True, sign_inputs=True)
+    ref = oracle.conv(x, wb.e, wb.alpha, wb.beta, c["kh"], c["kw"], c["stride"], c["pad"], sign_inputs=True)
+    n = w.shape[1]
+    assert np.array_equal(det.pK.cpu().numpy(), ref.p_K) and np.array_equal(unpack(words(det.pmask), n), ref.p_e)
+    assert rel_close(det.pgamma.cpu().numpy(), ref.p_gamma).all() and rel_close(det.pdelta.cpu().numpy(), ref.p_delta).all()
+    assert np.array_equal(det.p11.cpu().numpy(), ref.p_p11)
+    # gamma may differ in the last bit (summation order), so the outputs are compared within the tolerance
+    assert rel_close(y.cpu().numpy(), ref.y, 2e-5).all()
+
+
 @pytest.mark.parametrize("batch", [1, 2, 19])
 def test_conv_host_entry_point(dab, batch):
     # host tensors in and out; the batch is pipelined in chunks (19 images: 7 chunks, the last one ragged)
