@@ -301,15 +301,24 @@ static void set_tile(const dab_conv_desc& d, int Ho, int Wo, const int (&sh)[2],
   a->magic_in_w = in_w > 1 ? (uint32_t)((two32 + (uint64_t)in_w - 1) / (uint64_t)in_w) : 0u;
 }
 
-// Picks the tile and launches.  The largest tile is taken that still lets at least 16 warps be resident per SM
-// (shared memory is the limit); if no shape reaches that, the shape with the most resident CTAs wins.
+// Picks the tile and launches.  A shape is admissible if its staged input fits and it leaves 16 to 24 warps
+// resident per SM (shared memory is the limit); `groups` = patches a CTA codes at a time.  Among the admissible
+// shapes the largest one that still gives two CTAs per SM of work is taken (large layers: least halo re-reading);
+// a small layer, which cannot fill the GPU with large tiles, gets the smallest shape that keeps all groups of a
+// CTA busy (most CTAs, shortest critical path).  If nothing is admissible the shape with the most resident CTAs wins.
 template <typename Kernel>
-static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes, int threads, cudaStream_t stream) {
+static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes, int threads, int groups,
+                                  cudaStream_t stream) {
   const size_t sm_bytes = 228 * 1024, cta_reserve = 1024, cta_limit = 227 * 1024;
-  const int want_ctas = (16 * 32 + threads - 1) / threads;
-  int best = -1, best_ctas = 0;
-  size_t best_smem = 0;
-  for (int i = 0; i < (int)(sizeof(kTileShapes) / sizeof(kTileShapes[0])); ++i) {
+  // resident warps per SM a shape must leave room for: measured best is 24 for one or two warps per patch (their
+  // tile loads overlap other CTAs' sorting), 16 for larger groups (fewer, larger tiles matter more)
+  const int want_warps = groups >= 4 ? 24 : 16;
+  const int want_ctas = (want_warps * 32 + threads - 1) / threads;
+  const int64_t want_tiles = 2 * 148;
+  int best = -1, best_ctas = 0, small = -1;
+  size_t best_smem = 0, small_smem = 0;
+  bool settled = false;
+  for (int i = 0; i < (int)(sizeof(kTileShapes) / sizeof(kTileShapes[0])) && !settled; ++i) {
     if (a.tile_shape >= 0 && i != a.tile_shape) continue;
     PatchArgs t = a;
     set_tile(a.d, a.Ho, a.Wo, kTileShapes[i], &t);
@@ -320,8 +329,14 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
     int ctas = (int)(sm_bytes / (smem + cta_reserve));
     if (ctas > 2048 / threads) ctas = 2048 / threads;
     if (ctas > best_ctas) { best = i; best_ctas = ctas; best_smem = smem; }
-    if (ctas >= want_ctas) break;
+    if (ctas >= want_ctas) {
+      const int64_t tiles = (int64_t)t.tiles_h * t.tiles_w * a.d.N;
+      const bool busy = t.TH * t.TW >= groups;  // every group of the CTA has a patch
+      if ((tiles >= want_tiles && busy) || a.tile_shape >= 0) { best = i; best_smem = smem; settled = true; }
+      else if (busy || small < 0) { small = i; small_smem = smem; }
+    }
   }
+  if (!settled && small >= 0) { best = small; best_smem = small_smem; }
   if (best < 0) return cudaErrorInvalidValue;
   a.tile_shape = best;
   set_tile(a.d, a.Ho, a.Wo, kTileShapes[best], &a);
@@ -336,7 +351,7 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
 template <int R, bool kFull>
 static cudaError_t launch_patches_warp(PatchArgs& a, cudaStream_t stream) {
   size_t fixed = sizeof(double) * rcp_table_slots(a.n) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
-  return launch_patches(binarize_patches_warp_kernel<R, kFull>, a, fixed, kWarpsPerCta * 32, stream);
+  return launch_patches(binarize_patches_warp_kernel<R, kFull>, a, fixed, kWarpsPerCta * 32, kWarpsPerCta, stream);
 }
 
 template <int W, int WARPS, int R, bool kFull, bool kTable>
@@ -345,7 +360,7 @@ static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream) {
   a.scratch_words = scratch_words_for(a.n, W);
   size_t fixed = (kTable ? sizeof(double) * rcp_table_slots(a.n) : 0) + sizeof(GroupShared) * G +
                  sizeof(uint32_t) * (size_t)a.scratch_words * G;
-  return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, stream);
+  return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, G, stream);
 }
 
 cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
@@ -356,7 +371,7 @@ cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, 
   a.scratch_words = 0;
   a.defer_dense = 0; a.marked_only = 0; a.tile_shape = -1;
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
-  return launch_patches(sign_patches_kernel, a, 0, kWarpsPerCta * 32, stream);
+  return launch_patches(sign_patches_kernel, a, 0, kWarpsPerCta * 32, kWarpsPerCta, stream);
 }
 
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
