@@ -22,9 +22,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
 
   for (int64_t row = (int64_t)blockIdx.x * kWarpsPerCta + warp; row < rows; row += (int64_t)gridDim.x * kWarpsPerCta) {
     const float* v = values + row * ld_values;
-    auto value = [v](int i) { return __ldg(v + i); };
+    auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
     uint32_t kreg[R];
-    RowResult res = warp_code_row<R, kFull>(value, n, lane, scratch, rcp, kreg);
+    RowResult res = warp_code_row<R, kFull>(keyof, n, lane, scratch, rcp, kreg);
     if (lane == 0) {
       K_out[row] = res.K;
       alpha_out[row] = res.alpha;
@@ -63,9 +63,9 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
 
   for (int64_t row = (int64_t)blockIdx.x * G + group; row < rows; row += (int64_t)gridDim.x * G) {
     const float* v = values + row * ld_values;
-    auto value = [v](int i) { return __ldg(v + i); };
+    auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
     uint32_t kreg[R];
-    group_code_row<W, R, kFull, kTable>(value, n, tig, scratch, gs, bar_id, rcp, kreg);
+    group_code_row<W, R, kFull, kTable>(keyof, n, tig, scratch, gs, bar_id, rcp, kreg);
     const RowResult res = gs->result;
     if (tig == 0) {
       K_out[row] = res.K;

@@ -39,7 +39,9 @@ __device__ __forceinline__ void fill_offsets(const PatchArgs& a, uint16_t* off, 
 }
 
 // Stages the tile whose first input row/column is (h0, w0) of image `ximg`; out-of-image positions become 0.0.
-// Returns the number of non-zero values this thread staged.
+// Returns the number of non-zero values this thread staged.  kKeys: the tile holds the order-preserving keys of the
+// values (each element is part of up to kh*kw patches: its key is computed once here, not once per patch).
+template <bool kKeys>
 __device__ __forceinline__ int load_tile(const PatchArgs& a, const float* __restrict__ ximg, int h0, int w0,
                                          float* tile, int ch_words, int tid, int threads) {
   const int per_ch = a.in_h * a.in_w;
@@ -54,7 +56,7 @@ __device__ __forceinline__ int load_tile(const PatchArgs& a, const float* __rest
     float v = 0.0f;
     if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
       v = __ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w);
-    tile[c * ch_words + r * a.pitch + s] = v;
+    tile[c * ch_words + r * a.pitch + s] = kKeys ? __uint_as_float(order_key(v)) : v;
     nonzero += (v != 0.0f);
   }
   return nonzero;
@@ -107,7 +109,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
     const TileCoord t = tile_coord(a, tile_id);
     __syncthreads();  // the previous tile is no longer read
     if (threadIdx.x == 0) tile_nonzero = 0;
-    int nz = load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x,
+    int nz = load_tile<true>(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x,
                        THREADS);
     const int64_t first_patch = ((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0;
     if (a.defer_dense) {
@@ -130,9 +132,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
     for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
       const int lh = p / t.tw, lw = p % t.tw;
       const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
-      auto value = [origin, off](int i) { return origin[off[i]]; };
+      auto keyof = [origin, off](int i) { return __float_as_uint(origin[off[i]]); };
       uint32_t kreg[R];
-      RowResult res = warp_code_row<R, kFull>(value, a.n, lane, scratch, rcp, kreg);
+      RowResult res = warp_code_row<R, kFull>(keyof, a.n, lane, scratch, rcp, kreg);
       const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
       if (lane == 0) {
         a.pK[pi] = res.K;
@@ -172,15 +174,15 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
     const TileCoord t = tile_coord(a, tile_id);
     if (a.marked_only && a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] != kDenseMark) continue;
     __syncthreads();
-    load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
+    load_tile<true>(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
     __syncthreads();
 
     for (int p = group; p < t.th * t.tw; p += G) {
       const int lh = p / t.tw, lw = p % t.tw;
       const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
-      auto value = [origin, off](int i) { return origin[off[i]]; };
+      auto keyof = [origin, off](int i) { return __float_as_uint(origin[off[i]]); };
       uint32_t kreg[R];
-      group_code_row<W, R, kFull, kTable>(value, a.n, tig, scratch, gs, bar_id, rcp, kreg);
+      group_code_row<W, R, kFull, kTable>(keyof, a.n, tig, scratch, gs, bar_id, rcp, kreg);
       const RowResult res = gs->result;
       const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
       if (tig == 0) {
@@ -251,7 +253,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) sign_patches_kernel(const P
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
     __syncthreads();
-    load_tile(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
+    load_tile<false>(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
     __syncthreads();
     for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
       const int lh = p / t.tw, lw = p % t.tw;

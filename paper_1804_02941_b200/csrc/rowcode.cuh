@@ -451,12 +451,12 @@ __device__ __noinline__ void group_sort_select(uint32_t* scratch, int m, int z, 
   if (tig == 0) gs->result = res;
 }
 
-// Codes one row with a group of W > 1 warps.  `value(i)` returns element i (0 <= i < n).  Warp w of the group
+// Codes one row with a group of W > 1 warps.  `keyof(i)` returns the order-preserving key of element i (0 <= i < n).  Warp w of the group
 // owns rounds w*R .. w*R+R-1 of the row (element (round)*32 + lane) and keeps their keys in kreg[], so that the
 // mask needs no second read of the values.  kFull: n == 32*W*R exactly.  On return gs->result is valid for
 // every thread of the group.
-template <int W, int R, bool kFull, bool kTable, typename Value>
-__device__ __forceinline__ void group_code_row(Value value, int n, int tig, uint32_t* scratch, GroupShared* gs,
+template <int W, int R, bool kFull, bool kTable, typename KeyOf>
+__device__ __forceinline__ void group_code_row(KeyOf keyof, int n, int tig, uint32_t* scratch, GroupShared* gs,
                                                int bar_id, const double* rcp, uint32_t (&kreg)[R]) {
   static_assert(W > 1, "single warps use warp_code_row");
   constexpr int GT = 32 * W;
@@ -471,7 +471,7 @@ __device__ __forceinline__ void group_code_row(Value value, int n, int tig, uint
     uint32_t key = kZeroKey;
     const int i = first + k * 32;
     if (kFull || i < n) {
-      key = order_key(value(i));
+      key = keyof(i);
       kmin = min(kmin, key);
       kmax = max(kmax, key);
     }
@@ -566,8 +566,8 @@ __device__ __noinline__ RowResult warp_sort_select_outlined(const uint32_t* scra
 
 // Returns the result in every lane.  scratch: 32*R words of shared memory owned by the warp; rcp: n+1 reciprocals.
 // kFull: n == 32*R exactly (no bounds tests in the load loop).
-template <int R, bool kFull, typename Value>
-__device__ __forceinline__ RowResult warp_code_row(Value value, int n, int lane, uint32_t* scratch,
+template <int R, bool kFull, typename KeyOf>
+__device__ __forceinline__ RowResult warp_code_row(KeyOf keyof, int n, int lane, uint32_t* scratch,
                                                    const double* rcp, uint32_t (&kreg)[R]) {
   const unsigned lt = (1u << lane) - 1u;
   uint32_t kmin = kPadKey, kmax = 0u;
@@ -578,7 +578,7 @@ __device__ __forceinline__ RowResult warp_code_row(Value value, int n, int lane,
     if (kFull || k * 32 < n) {
       const int i = k * 32 + lane;
       if (kFull || i < n) {
-        key = order_key(value(i));
+        key = keyof(i);
         kmin = min(kmin, key);
         kmax = max(kmax, key);
       }
