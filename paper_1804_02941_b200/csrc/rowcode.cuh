@@ -287,7 +287,7 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
       for (int w = 0; w < W; ++w) gmax = fmax(gmax, gs->wmax[w]);
     }
     const double thr = gmax * kBand;
-    unsigned cmask = (Dz >= thr) ? (1u << E) : 0u;
+    unsigned cmask = (Dz >= thr) ? (1u << (E & 31)) : 0u;  // this branch exists for E <= 8 only
 #pragma unroll
     for (int j = 0; j < E; ++j) cmask |= (Dj[kKeep ? j : 0] >= thr) ? (1u << j) : 0u;
     int total = __reduce_add_sync(0xFFFFFFFFu, __popc(cmask));
