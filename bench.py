@@ -32,10 +32,10 @@ SM_COUNT = 148
 # dram__bytes_read.sum + dram__bytes_write.sum of the patch-coder launches of each layer at batch 256, from one
 # ncu capture of this benchmark (profiles/binarize_patches_dram_traffic_config5.md).  Valid for the kernels as
 # they were then: reset to {} when the patch coder changes.
-PATCH_CODER_DRAM_BYTES = {"l1_0": 274342912, "l1_1": 270581760, "l1_2": 272141056, "l1_3": 271047936, "l2_0": 221521408,
-                          "l2_1": 120040960, "l2_2": 119217920, "l2_3": 119235584, "l3_0": 107264000, "l3_1": 52955136,
-                          "l3_2": 53775104, "l3_3": 53685760, "l4_0": 52193280, "l4_1": 26870272, "l4_2": 26882304,
-                          "l4_3": 26891008}
+PATCH_CODER_DRAM_BYTES = {"l1_0": 275064576, "l1_1": 271620608, "l1_2": 272581632, "l1_3": 272041216, "l2_0":
+                          222675712, "l2_1": 119762688, "l2_2": 120052736, "l2_3": 119627776, "l3_0": 106836736,
+                          "l3_1": 52807680, "l3_2": 53128448, "l3_3": 52924928, "l4_0": 52207872, "l4_1": 26969344,
+                          "l4_2": 26978816, "l4_3": 26957568}
 
 
 def parse_args():
