@@ -40,9 +40,6 @@ __device__ __forceinline__ void group_barrier(int bar_id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(threads) : "memory");
 }
 
-// Index skew for scratch arrays read with a stride of E words between lanes (E a power of two up to 32).
-__device__ __forceinline__ int skew(int i) { return i + (i >> 5); }
-
 // Ascending bitonic sort of 32*W*E keys, E per thread, blocked layout.
 template <int W, int E>
 __device__ __forceinline__ void group_sort(uint32_t (&r)[E], int tig, uint32_t* xbuf, int bar_id) {

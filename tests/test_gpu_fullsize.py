@@ -93,6 +93,29 @@ def test_config5_layers_at_batch_256(dab, name):
     _check_layer(dab, L, stream=7)
 
 
+def test_config5_first_layer_sign_coded_inputs(dab):
+    # the XNOR-style input coding at full size: sampled patches against the checker
+    L = configs.config5(256)[0]
+    x = L.inputs(stream=9, dense=True)
+    w = L.weights(stream=9)
+    xd, wd, wb = to_dev(x), dab.dab_binarize(to_dev(w)), oracle.binarize(w)
+    y, det = dab.dab_binary_conv(xd, wd, 3, 3, (1, 1), (1, 1), details=True, sign_inputs=True)
+    torch.cuda.synchronize()
+    P = L.patches
+    idx = np.unique(np.concatenate([[0, L.Wo - 1, P - 1], (dab_synth.uniform01(97, 1, 0, 160) * P).astype(np.int64)]))
+    ref = oracle.sign_code(_sample_patches(x, L, idx))
+    t = torch.from_numpy(idx).to(xd.device)
+    assert np.array_equal(det.pK[t].cpu().numpy(), ref.K) and np.array_equal(unpack(words(det.pmask[t]), L.n), ref.e)
+    assert rel_close(det.pgamma[t].cpu().numpy(), ref.alpha).all()
+    refC, refP = oracle.gemm(ref.e, ref.alpha, ref.beta, wb.e, wb.alpha, wb.beta)
+    assert np.array_equal(det.p11[t].cpu().numpy(), refP)
+    img, rem = np.divmod(idx, L.Ho * L.Wo)
+    ho, wo = np.divmod(rem, L.Wo)
+    dev = xd.device
+    got = y[torch.from_numpy(img).to(dev), :, torch.from_numpy(ho).to(dev), torch.from_numpy(wo).to(dev)].cpu().numpy()
+    assert rel_close(got, refC, 2e-5).all()
+
+
 def test_config5_first_layer_dense_inputs(dab):
     L = configs.config5(64)[0]
     _check_layer(dab, L, stream=8, dense=True)
