@@ -173,7 +173,7 @@ dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, con
 
 /*
  * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up
- * to 8 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
+ * to 16 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
  * chunks overlap on three streams, and the call returns after everything has drained.  Use pinned host memory:
  * with pageable memory the copies are staged by the driver and do not overlap.  The two copy streams and a few
  * events are created on the first call on a device and kept for the life of the process (the only state the

@@ -238,7 +238,7 @@ dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, con
 // ---------------------------------------------------------------------------------------------------------
 namespace {
 
-constexpr int kHostChunks = 8;  // chunks per call at most
+constexpr int kHostChunks = 16;  // chunks per call at most
 
 struct HostPipe {
   bool ready = false;

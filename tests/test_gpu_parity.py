@@ -242,7 +242,7 @@ def test_conv_with_sign_coded_inputs_matches_checker(dab, ci):
 
 @pytest.mark.parametrize("batch", [1, 2, 19])
 def test_conv_host_entry_point(dab, batch):
-    # host tensors in and out; the batch is pipelined in chunks (19 images: 7 chunks, the last one ragged)
+    # host tensors in and out; the batch is pipelined in chunks (19 images: 10 chunks of 2, the last one ragged)
     L = configs.ConvLayer("t", batch, 16, 12, 12, 24, 3, 3, 1, 1)
     x, w = L.inputs(stream=5), L.weights(stream=5)
     wd = dab.dab_binarize(to_dev(w))
