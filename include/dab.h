@@ -212,6 +212,28 @@ dab_status dab_binary_conv_static(const dab_conv_desc* desc, const float* d_x, c
                                   void* stream);
 
 /*
+ * Which kernel forms the AND-popcounts of dab_binary_gemm and of every convolution entry point (Section 4.2
+ * counts set bits with population-count instructions; an AND-popcount over n bits is also the dot product of
+ * the two rows written as 0/1 bytes, which the tensor cores form exactly in 32-bit integers):
+ *   DAB_CONTRACT_TENSOR  (default) mask words are expanded to bytes in shared memory and multiplied by
+ *                        tcgen05.mma kind::i8 into tensor memory;
+ *   DAB_CONTRACT_POPC    AND, carry-save adders and population counts on the integer pipes.
+ * Both give the same counts bit for bit and apply the same four-term rescale.  The setting is process-wide and
+ * read at each call; it exists so that the two can be measured against each other.
+ */
+typedef enum { DAB_CONTRACT_TENSOR = 0, DAB_CONTRACT_POPC = 1 } dab_contraction;
+dab_status dab_set_contraction(dab_contraction path);
+dab_contraction dab_get_contraction(void);
+
+/*
+ * The tensor-core kernel waits on hardware barriers with a time limit (about two seconds) instead of
+ * forever; a wait that ran out is counted on the device and leaves that tile's outputs unwritten.
+ * dab_contraction_wait_failures copies the current device's count since library load to *h_count (host
+ * pointer).  Synchronises the device.  0 on every correct run.
+ */
+dab_status dab_contraction_wait_failures(uint32_t* h_count);
+
+/*
  * dab_popc_probe — measurement aid, not part of the method: runs `iters` rounds of independent
  * AND + population-count + add chains in every thread of a grid of `blocks` x 256 threads and
  * writes one word per thread to d_sink (blocks*256 words), so that a caller timing it obtains the

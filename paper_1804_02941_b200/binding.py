@@ -23,7 +23,8 @@ ROW_NONFINITE = 2
 EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_binarize", "dab_pack", "dab_binary_gemm",
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
-           "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe")
+           "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures")
 
 
 class DabError(RuntimeError):
@@ -70,6 +71,9 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_static_capacity.argtypes = []
         L.dab_binary_conv_static.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
+        L.dab_set_contraction.argtypes = [i32]
+        L.dab_get_contraction.argtypes = []
+        L.dab_contraction_wait_failures.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -320,3 +324,22 @@ def dab_popc_probe(blocks: int, iters: int, sink: torch.Tensor | None = None, st
         sink = torch.empty(blocks * 256, dtype=torch.int32, device="cuda")
     _check(lib().dab_popc_probe(_ptr(sink), blocks, iters, _stream(stream)), "dab_popc_probe")
     return sink
+
+
+CONTRACT_TENSOR, CONTRACT_POPC = 0, 1
+
+
+def dab_set_contraction(path: int) -> None:
+    """Process-wide choice of the contraction kernel: CONTRACT_TENSOR (default) or CONTRACT_POPC."""
+    _check(lib().dab_set_contraction(int(path)), "dab_set_contraction")
+
+
+def dab_get_contraction() -> int:
+    return int(lib().dab_get_contraction())
+
+
+def dab_contraction_wait_failures() -> int:
+    """Barrier waits of the tensor-core kernel that ran out on the current device (0 on a correct run)."""
+    c = C.c_uint32(0)
+    _check(lib().dab_contraction_wait_failures(C.byref(c)), "dab_contraction_wait_failures")
+    return int(c.value)

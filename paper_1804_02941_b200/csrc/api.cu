@@ -1,5 +1,6 @@
 // C ABI of libdab: argument validation on the host, then launches.  No device memory is allocated; the only
 // state kept is the pair of copy streams of the host-buffer convolution.
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -13,6 +14,18 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline dab_status from_cuda(cudaError_t e) { return e == cudaSuccess ? DAB_OK : DAB_ERR_CUDA; }
 
 constexpr size_t kAlign = 256;
+
+std::atomic<int> g_contraction{(int)DAB_CONTRACT_TENSOR};
+
+// The contraction kernel the process-wide setting names.  The tensor-core kernel tiles the column side
+// (weights when lanes_along_rows, activations otherwise) 256 rows per grid row; a launch too tall for
+// that takes the population-count kernel.
+cudaError_t contract(const GemmArgs& g, bool lanes_along_rows, cudaStream_t stream) {
+  const int64_t column_rows = lanes_along_rows ? g.N : g.M;
+  if (g_contraction.load(std::memory_order_relaxed) == (int)DAB_CONTRACT_TENSOR && column_rows <= (int64_t)65535 * 256)
+    return launch_gemm_mma(g, lanes_along_rows, stream);
+  return launch_gemm(g, lanes_along_rows, stream);
+}
 
 struct ConvGeom {
   int32_t Ho, Wo, n, ld;
@@ -110,7 +123,7 @@ dab_status dab_binary_gemm(int64_t M, int64_t N, int32_t n, const uint32_t* d_A,
   g.C = d_C;
   g.map.inner = M; g.map.outer_stride = 0; g.map.row_stride = ldc; g.map.col_stride = 1;
   g.p11 = d_p11; g.ldp = ldp;
-  return from_cuda(launch_gemm(g, /*lanes_along_rows=*/false, static_cast<cudaStream_t>(stream)));
+  return from_cuda(contract(g, /*lanes_along_rows=*/false, static_cast<cudaStream_t>(stream)));
 }
 
 dab_status dab_conv_output_size(const dab_conv_desc* desc, int32_t* Ho, int32_t* Wo) {
@@ -184,7 +197,7 @@ dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d
   int64_t HoWo = (int64_t)g.Ho * g.Wo;
   a.map.inner = HoWo; a.map.outer_stride = (int64_t)desc->Cout * HoWo; a.map.row_stride = 1; a.map.col_stride = HoWo;
   a.p11 = d_p11; a.ldp = desc->Cout;
-  return from_cuda(launch_gemm(a, /*lanes_along_rows=*/true, static_cast<cudaStream_t>(stream)));
+  return from_cuda(contract(a, /*lanes_along_rows=*/true, static_cast<cudaStream_t>(stream)));
 }
 
 static dab_status conv_with_coder(bool sign, const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
@@ -352,6 +365,22 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
   cudaError_t e1 = cudaStreamSynchronize(hp->in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(hp->out);
   if (status != DAB_OK) return status;
   return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess) ? DAB_OK : DAB_ERR_CUDA;
+}
+
+dab_status dab_set_contraction(dab_contraction path) {
+  if (path != DAB_CONTRACT_TENSOR && path != DAB_CONTRACT_POPC) return DAB_ERR_INVALID_ARG;
+  g_contraction.store((int)path, std::memory_order_relaxed);
+  return DAB_OK;
+}
+
+dab_contraction dab_get_contraction(void) { return (dab_contraction)g_contraction.load(std::memory_order_relaxed); }
+
+dab_status dab_contraction_wait_failures(uint32_t* h_count) {
+  if (!h_count) return DAB_ERR_INVALID_ARG;
+  unsigned int c = 0;
+  cudaError_t e = read_mma_wait_timeouts(&c);
+  *h_count = c;
+  return from_cuda(e);
 }
 
 dab_status dab_popc_probe(uint32_t* d_sink, int32_t blocks, int32_t iters, void* stream) {

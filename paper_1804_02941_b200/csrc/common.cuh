@@ -37,6 +37,21 @@ __device__ __forceinline__ double objective(double P, double T, int s, int n) {
   return __dadd_rn(__ddiv_rn(__dmul_rn(P, P), (double)s), __ddiv_rn(__dmul_rn(Q, Q), (double)(n - s)));
 }
 
+// Exact int32 -> fp64 without the conversion unit: 2^52 + 2^31 + p has p ^ 0x80000000 as its low word.
+__device__ __forceinline__ double int_to_double(int p) {
+  return __hiloint2double(0x43300000, (int)((unsigned)p ^ 0x80000000u)) - 4503601774854144.0;
+}
+
+// Four-term rescale in fp64, one rounding to fp32.  Term order is part of the contract.
+__device__ __forceinline__ float rescale(int p11, int Ke, int Kf, int n, double a, double b, double g, double d) {
+  int p10 = Ke - p11, p01 = Kf - p11, p00 = n - Ke - Kf + p11;
+  double y = __dmul_rn(__dmul_rn(a, g), int_to_double(p11));
+  y = __dadd_rn(y, __dmul_rn(__dmul_rn(a, d), int_to_double(p10)));
+  y = __dadd_rn(y, __dmul_rn(__dmul_rn(b, g), int_to_double(p01)));
+  y = __dadd_rn(y, __dmul_rn(__dmul_rn(b, d), int_to_double(p00)));
+  return (float)y;
+}
+
 // Where an output element (row i of the activation side, column j of the weight side) is stored:
 //   offset = (i / inner) * outer_stride + (i % inner) * row_stride + j * col_stride
 // Row-major M x N: inner = M (never wraps), row_stride = ldc, col_stride = 1.
@@ -70,6 +85,9 @@ cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_
 cudaError_t launch_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld_bits, uint32_t* mask,
                         int32_t ld_mask, int32_t* K, cudaStream_t stream);
 cudaError_t launch_gemm(const GemmArgs& args, bool lanes_along_rows, cudaStream_t stream);
+// Tensor-core contraction; lanes_along_rows as for launch_gemm.  See gemm_mma.cu.
+cudaError_t launch_gemm_mma(const GemmArgs& args, bool lanes_along_rows, cudaStream_t stream);
+cudaError_t read_mma_wait_timeouts(unsigned int* count);
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
                                     float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
                                     cudaStream_t stream);

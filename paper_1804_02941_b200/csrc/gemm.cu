@@ -10,21 +10,6 @@ constexpr int TM = 4, TN = 4;    // outputs per thread
 constexpr int GEMM_THREADS = 256;
 constexpr int SLD = BM + 4;      // padded smem row, keeps 16-byte alignment
 
-// Exact int32 -> fp64 without the conversion unit: 2^52 + 2^31 + p has p ^ 0x80000000 as its low word.
-__device__ __forceinline__ double int_to_double(int p) {
-  return __hiloint2double(0x43300000, (int)((unsigned)p ^ 0x80000000u)) - 4503601774854144.0;
-}
-
-// Four-term rescale in fp64, one rounding to fp32.  Term order is part of the contract.
-__device__ __forceinline__ float rescale(int p11, int Ke, int Kf, int n, double a, double b, double g, double d) {
-  int p10 = Ke - p11, p01 = Kf - p11, p00 = n - Ke - Kf + p11;
-  double y = __dmul_rn(__dmul_rn(a, g), int_to_double(p11));
-  y = __dadd_rn(y, __dmul_rn(__dmul_rn(a, d), int_to_double(p10)));
-  y = __dadd_rn(y, __dmul_rn(__dmul_rn(b, g), int_to_double(p01)));
-  y = __dadd_rn(y, __dmul_rn(__dmul_rn(b, d), int_to_double(p00)));
-  return (float)y;
-}
-
 // Population counts issue at a quarter of the rate of logic operations, so three AND-ed words are first
 // compressed by a carry-save adder (two 3-input logic operations) into a sum word and a carry word:
 // popc(x0) + popc(x1) + popc(x2) = popc(sum) + 2 popc(carry).  Two counts instead of three.

@@ -1,0 +1,342 @@
+// Tensor-core form of the AND-popcount contraction (Section 4.2: the four population counts of a pair of
+// coded rows).  popc(e AND f) over a row of n bits is the dot product of the two rows written as 0/1 bytes,
+// so each CTA expands mask words to bytes in shared memory and lets the fifth-generation tensor cores
+// (tcgen05.mma, kind::i8, unsigned 8-bit operands, 32-bit integer accumulators in tensor memory) form a
+// 128 x NT block of exact integer counts.  The four-term rescale then runs on the counts as they are read
+// back from tensor memory, with the same arithmetic as the population-count kernel.
+//
+// Shared-memory operand layout (K-major, no swizzle): 8 rows x 16 bytes form one contiguous 128-byte core
+// matrix; core matrices of consecutive 16-byte K chunks follow each other (leading byte offset 128) and
+// groups of 8 rows are one whole stage row apart (stride byte offset = K chunks per stage x 128).  One mask
+// word is 32 K bytes = two K chunks = the K extent of one kind::i8 instruction.
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace dab {
+namespace {
+
+constexpr int MMA_M = 128;       // activation rows per CTA = lanes of tensor memory
+constexpr int MMA_NMAX = 256;    // weight rows per CTA = columns of tensor memory
+constexpr int MMA_THREADS = 256;
+constexpr int MMA_STAGES = 2;
+constexpr long long kWaitCycles = 4000000000ll;  // about two seconds; a wait that long has failed
+
+__device__ unsigned int g_mma_wait_timeouts;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Shared-memory matrix descriptor: address, leading and stride byte offsets in 16-byte units, descriptor
+// version 1 in bits [46,48), no swizzle (layout type 0 in bits [61,64)).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46);
+}
+
+// Instruction descriptor of kind::i8: D format S32 (2 at bit 4), A and B unsigned 8-bit (0 at bits 7 and 10),
+// both K-major (0 at bits 15 and 16), N / 8 at bit 17, M / 16 at bit 24.
+__device__ __forceinline__ uint32_t instr_desc(int nt) {
+  return (2u << 4) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+// Bounded wait for the phase with the given parity.  Returns false after kWaitCycles and counts the failure;
+// the caller then stops waiting on anything (dead stays set) but keeps its control flow, so that every
+// thread still reaches every barrier and the CTA ends.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, bool& dead) {
+  if (dead) return false;
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if (clock64() - t0 > kWaitCycles) {
+      dead = true;
+      atomicAdd(&g_mma_wait_timeouts, 1u);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void mma_i8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+      :
+      : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+      : "memory");
+}
+
+// Arrives on the barrier once every tcgen05.mma issued by this thread so far has completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Four mask bits -> four bytes of 0/1 (bit i to byte i): the products i + 7j land on distinct bit positions.
+__device__ __forceinline__ uint32_t spread4(uint32_t nibble) { return (nibble * 0x00204081u) & 0x01010101u; }
+
+// One 16-byte piece (four mask words) of one row -> eight 16-byte K chunks in the stage.
+// dst points at the row's slot in the K chunk of the first word; consecutive K chunks are 128 bytes apart.
+__device__ __forceinline__ void expand_words(uint4 q, unsigned char* dst) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int m = 0; m < 4; ++m) {
+    uint4 lo, hi;
+    lo.x = spread4(w[m] & 15u);
+    lo.y = spread4((w[m] >> 4) & 15u);
+    lo.z = spread4((w[m] >> 8) & 15u);
+    lo.w = spread4((w[m] >> 12) & 15u);
+    hi.x = spread4((w[m] >> 16) & 15u);
+    hi.y = spread4((w[m] >> 20) & 15u);
+    hi.z = spread4((w[m] >> 24) & 15u);
+    hi.w = spread4(w[m] >> 28);
+    *reinterpret_cast<uint4*>(dst + (2 * m) * 128) = lo;
+    *reinterpret_cast<uint4*>(dst + (2 * m + 1) * 128) = hi;
+  }
+}
+
+// One operand of the contraction: packed rows with their popcounts and the two reconstruction values
+// (gamma, delta on the activation side; alpha, beta on the weight side).
+struct Side {
+  const uint32_t* mask;
+  int32_t ld;
+  const int32_t* K;
+  const float* v1;  // value of the set bits
+  const float* v0;  // value of the clear bits
+  int64_t rows;
+};
+
+// The pieces one thread expands per stage: unit u covers row (u>>3)/KQ*8 + (u&7), 16-byte piece (u>>3)%KQ.
+// Eight consecutive lanes hold the eight rows of one core matrix, so their 16-byte stores are one
+// contiguous 128 bytes; their loads read KQ x 16 contiguous bytes per row.
+constexpr int kMaxUnits = 3;
+
+// kLanesAreActivations: the rows that ride the 128 lanes of tensor memory (and the threads of the epilogue)
+// are activation rows, the columns weight rows: coalesced stores when the output is contiguous along the
+// activation rows (NCHW).  Otherwise the roles are exchanged: coalesced for a row-major M x N output.
+template <int KQ, bool kLanesAreActivations>
+__global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const GemmArgs g) {
+  constexpr int KC = 8 * KQ;            // 16-byte K chunks per stage (two per mask word)
+  constexpr uint32_t SBO = KC * 128;    // bytes between groups of 8 rows
+  extern __shared__ __align__(128) unsigned char stage_mem[];
+  __shared__ double s_v1[MMA_NMAX], s_v0[MMA_NMAX];  // column side
+  __shared__ int64_t s_off[MMA_NMAX];
+  __shared__ int s_K[MMA_NMAX];
+  __shared__ __align__(8) uint64_t s_bar[MMA_STAGES];
+  __shared__ uint32_t s_tmem;
+
+  const Side act{g.A, g.lda, g.KA, g.gamma, g.delta, g.M}, wgt{g.B, g.ldb, g.KB, g.alpha, g.beta, g.N};
+  const Side L = kLanesAreActivations ? act : wgt;  // lane side
+  const Side S = kLanesAreActivations ? wgt : act;  // column side
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t i0 = (int64_t)blockIdx.x * MMA_M;
+  const int64_t j0 = (int64_t)blockIdx.y * MMA_NMAX;
+  const int nrows = (int)min((int64_t)MMA_NMAX, S.rows - j0);  // column-side rows of this tile
+  const int NT = (nrows + 15) & ~15;                            // instruction N
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < NT) tmem_cols <<= 1;
+
+  const uint32_t a_bytes = MMA_M * KC * 16;
+  const int ncap = (int)min((int64_t)MMA_NMAX, (S.rows + 15) & ~(int64_t)15);  // widest tile of this launch
+  const uint32_t stage_bytes = a_bytes + (uint32_t)ncap * KC * 16;
+  const uint32_t mem0 = (smem_u32(stage_mem) + 127u) & ~127u;
+  unsigned char* const mem0_ptr = stage_mem + (mem0 - smem_u32(stage_mem));
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < MMA_STAGES; ++s) mbar_init(smem_u32(&s_bar[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // where activation row i and weight row j meet in the output: act_offset(i) + j * col_stride
+  auto act_offset = [&](int64_t i) {
+    return (i / g.map.inner) * g.map.outer_stride + (i % g.map.inner) * g.map.row_stride;
+  };
+  for (int j = tid; j < MMA_NMAX; j += MMA_THREADS) {
+    const bool in = j < nrows;
+    s_v1[j] = in ? (double)S.v1[j0 + j] : 0.0;
+    s_v0[j] = in ? (double)S.v0[j0 + j] : 0.0;
+    s_K[j] = in ? S.K[j0 + j] : 0;
+    s_off[j] = !in ? 0 : kLanesAreActivations ? (j0 + j) * g.map.col_stride : act_offset(j0 + j);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+  const uint32_t idesc = instr_desc(NT);
+
+  // units of this thread: lane-side pieces first, then column-side pieces
+  const int l_units = MMA_M * KQ, units = l_units + NT * KQ;
+  const int chunks = (g.words + 4 * KQ - 1) / (4 * KQ);
+  uint4 q[kMaxUnits];
+
+  auto fetch = [&](int c) {  // the 16-byte pieces of chunk c, zero beyond the operands
+    const int w0 = c * 4 * KQ;
+#pragma unroll
+    for (int t = 0; t < kMaxUnits; ++t) {
+      const int u = tid + t * MMA_THREADS;
+      q[t] = make_uint4(0, 0, 0, 0);
+      if (u >= units) continue;
+      const bool isL = u < l_units;
+      const int v = isL ? u : u - l_units;
+      const int row = ((v >> 3) / KQ) * 8 + (v & 7), piece = (v >> 3) % KQ;
+      const int w = w0 + 4 * piece;
+      if (w >= g.words) continue;
+      if (isL) {
+        if (i0 + row < L.rows) q[t] = *reinterpret_cast<const uint4*>(L.mask + (i0 + row) * (int64_t)L.ld + w);
+      } else {
+        if (row < nrows) q[t] = *reinterpret_cast<const uint4*>(S.mask + (j0 + row) * (int64_t)S.ld + w);
+      }
+    }
+  };
+
+  bool dead = false;
+  uint32_t parity[MMA_STAGES] = {0, 0};
+  fetch(0);
+  for (int c = 0; c < chunks; ++c) {
+    const int s = c & 1;
+    unsigned char* const stage = mem0_ptr + s * stage_bytes;
+    if (c >= MMA_STAGES) {  // the instructions that read this stage two chunks ago have completed
+      mbar_wait(smem_u32(&s_bar[s]), parity[s], dead);
+      parity[s] ^= 1;
+    }
+#pragma unroll
+    for (int t = 0; t < kMaxUnits; ++t) {
+      const int u = tid + t * MMA_THREADS;
+      if (u >= units) continue;
+      const bool isL = u < l_units;
+      const int v = isL ? u : u - l_units;
+      const int group = (v >> 3) / KQ, piece = (v >> 3) % KQ;
+      unsigned char* dst =
+          stage + (isL ? 0u : a_bytes) + (uint32_t)group * SBO + (uint32_t)(8 * piece) * 128 + (v & 7) * 16;
+      expand_words(q[t], dst);
+    }
+    if (c + 1 < chunks) fetch(c + 1);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> tensor-core reads
+    __syncthreads();
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a_addr = mem0 + s * stage_bytes, b_addr = a_addr + a_bytes;
+      const int kw = min(4 * KQ, g.words - c * 4 * KQ);
+      for (int t = 0; t < kw; ++t)  // one mask word = 32 K bytes = two K chunks per instruction
+        mma_i8(tmem, smem_desc(a_addr + t * 256, 128, SBO), smem_desc(b_addr + t * 256, 128, SBO), idesc,
+               (c | t) != 0);
+      mma_commit(smem_u32(&s_bar[s]));
+    }
+  }
+  {  // the last commit covers every instruction issued before it
+    const int s = (chunks - 1) & 1;
+    mbar_wait(smem_u32(&s_bar[s]), parity[s], dead);
+  }
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // Epilogue: thread = lane-side row (a warp reads the 32 lanes of its quarter), 32 columns at a time.
+  {
+    const int64_t gl = i0 + (warp & 3) * 32 + lane;
+    const bool valid = gl < L.rows && !dead;
+    int Kl = 0;
+    double l1 = 0.0, l0 = 0.0;
+    int64_t off = 0;
+    if (valid) {
+      Kl = L.K[gl];
+      l1 = (double)L.v1[gl];
+      l0 = (double)L.v0[gl];
+      off = kLanesAreActivations ? act_offset(gl) : gl * g.map.col_stride;
+    }
+    for (int cb = warp >> 2; cb * 32 < NT; cb += 2) {
+      uint32_t v[32];
+      tmem_load_32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cb * 32), v);
+      if (!valid) continue;
+#pragma unroll
+      for (int jj = 0; jj < 32; ++jj) {
+        const int j = cb * 32 + jj;
+        if (j >= nrows) break;
+        const int p11 = (int)v[jj];
+        // rescale(p11, K of the weight row, K of the activation row, n, alpha, beta, gamma, delta)
+        g.C[off + s_off[j]] = kLanesAreActivations ? rescale(p11, s_K[j], Kl, g.n, s_v1[j], s_v0[j], l1, l0)
+                                                   : rescale(p11, Kl, s_K[j], g.n, l1, l0, s_v1[j], s_v0[j]);
+        if (g.p11) g.p11[kLanesAreActivations ? gl * g.ldp + j0 + j : (j0 + j) * g.ldp + gl] = p11;
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+}
+
+template <int KQ, bool kLanesAreActivations>
+cudaError_t launch_kq(const GemmArgs& args, dim3 grid, int ncap, cudaStream_t stream) {
+  const size_t smem_max = (size_t)MMA_STAGES * (MMA_M + MMA_NMAX) * (8 * KQ) * 16 + 128;
+  const size_t smem = (size_t)MMA_STAGES * (MMA_M + ncap) * (8 * KQ) * 16 + 128;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
+    e = cudaFuncSetAttribute(binary_gemm_mma_kernel<KQ, kLanesAreActivations>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  binary_gemm_mma_kernel<KQ, kLanesAreActivations><<<grid, MMA_THREADS, smem, stream>>>(args);
+  return cudaGetLastError();
+}
+
+template <bool kLanesAreActivations>
+cudaError_t launch_side(const GemmArgs& args, cudaStream_t stream) {
+  const int64_t lane_rows = kLanesAreActivations ? args.M : args.N, col_rows = kLanesAreActivations ? args.N : args.M;
+  const int64_t gx = (lane_rows + MMA_M - 1) / MMA_M, gy = (col_rows + MMA_NMAX - 1) / MMA_NMAX;
+  if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
+  const dim3 grid((unsigned)gx, (unsigned)gy);
+  const int ncap = (int)std::min<int64_t>(MMA_NMAX, (col_rows + 15) & ~(int64_t)15);
+  // Two CTAs per SM (so that one expands while the other's counts are rescaled) bound the stage size:
+  // eight mask words per stage for narrow column tiles, four otherwise.
+  return ncap <= 64 ? launch_kq<2, kLanesAreActivations>(args, grid, ncap, stream)
+                    : launch_kq<1, kLanesAreActivations>(args, grid, ncap, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_mma(const GemmArgs& args, bool lanes_along_rows, cudaStream_t stream) {
+  if (args.words < 1 || args.M < 1 || args.N < 1) return cudaErrorInvalidValue;
+  return lanes_along_rows ? launch_side<true>(args, stream) : launch_side<false>(args, stream);
+}
+
+cudaError_t read_mma_wait_timeouts(unsigned int* count) {
+  return cudaMemcpyFromSymbol(count, g_mma_wait_timeouts, sizeof(unsigned int));
+}
+
+}  // namespace dab
