@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--dense", action="store_true", help="N(0,1) inputs without zeros instead of post-ReLU inputs")
     ap.add_argument("--layers", default="", help="comma-separated layer names (e.g. l1_0,l4_1) to run a subset; "
                     "the default is the whole workload")
+    ap.add_argument("--contraction", default="tensor", choices=["tensor", "popc"],
+                    help="contraction kernel: tcgen05 tensor cores on byte-expanded masks (default) or AND + population counts")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -62,6 +64,16 @@ def load_peaks():
             d = json.load(f)
         return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)", float(d.get("sm_max_mhz", 1965.0))
     return 6650.0, "fallback (earlier measurement on this pool)", 1965.0
+
+
+def load_int8_peak():
+    """Dense int8 tensor peak in TOPS: the measured sustained bf16 GEMM rate x the nominal int8:bf16 ratio (4.5 : 2.25)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return 2.0 * float(d["bf16_tflops_sustained"]), "2 x measured sustained bf16 GEMM rate (MEASURED_PEAKS.json)"
+    return 2.0 * 1400.0, "2 x fallback sustained bf16 GEMM rate"
 
 
 class ClockSampler:
@@ -226,6 +238,7 @@ def run_dab(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     dab.lib()
+    dab.dab_set_contraction(dab.CONTRACT_TENSOR if args.contraction == "tensor" else dab.CONTRACT_POPC)
     hbm_peak, peak_src, sm_max_mhz = load_peaks()
 
     layers = select_layers(configs.config5(args.batch), args)
@@ -338,13 +351,22 @@ def run_dab(args):
     contract_tops = ops_per_step * args.steps / (k_ms["contract"] * 1e-3) / 1e12
     popc_peak_measured = probe_words * 64 / 1e12     # plain AND+POPC+IADD chains: one count per word
     popc_peak_derived = POPC_PER_CLK_PER_SM * WORDS_PER_POPC * SM_COUNT * sm_max_mhz * 1e6 * 64 / 1e12
-    roofline_contract = {"kernel": "binary_gemm_kernel", "bound": "alu", "achieved": contract_tops,
-                         "peak": popc_peak_derived, "unit": "TOPS-equiv", "frac": contract_tops / popc_peak_derived,
-                         "plain_popc_rate_measured_by_probe": popc_peak_measured,
-                         "peak_source": "16 popc/clk/SM x 1.5 words per popc (3:2 carry-save) x 148 SMs x %.0f MHz x 64 binary "
-                                        "ops per word" % sm_max_mhz,
-                         "avg_launch_ms": k_ms["contract"] / launches_per_kind,
-                         "share_of_step": k_ms["contract"] / sum(k_ms.values())}
+    store_gbs = sum(4 * L.patches * L.Cout for L in layers) * args.steps / (k_ms["contract"] * 1e-3) / 1e9
+    common = {"achieved": contract_tops, "unit": "TOPS-equiv", "avg_launch_ms": k_ms["contract"] / launches_per_kind,
+              "share_of_step": k_ms["contract"] / sum(k_ms.values()), "output_store_gbs": store_gbs,
+              "output_store_frac_of_hbm": store_gbs / hbm_peak}
+    if args.contraction == "tensor":
+        int8_peak, int8_src = load_int8_peak()
+        roofline_contract = {"kernel": "binary_gemm_mma_kernel", "bound": "tensor", "peak": int8_peak,
+                             "frac": contract_tops / int8_peak, "peak_source": int8_src,
+                             "note": "kind::i8 on 0/1 bytes; the kernel's time goes to expanding mask words to bytes, the fp64 "
+                                     "rescale of every count and the output store, not to the tensor pipe", **common}
+    else:
+        roofline_contract = {"kernel": "binary_gemm_kernel", "bound": "alu", "peak": popc_peak_derived,
+                             "frac": contract_tops / popc_peak_derived,
+                             "plain_popc_rate_measured_by_probe": popc_peak_measured,
+                             "peak_source": "16 popc/clk/SM x 1.5 words per popc (3:2 carry-save) x 148 SMs x %.0f MHz x 64 "
+                                            "binary ops per word" % sm_max_mhz, **common}
 
     # end to end: host tensors in pinned memory, copies inside the timed region, through the host entry point
     e2e = None
@@ -384,12 +406,13 @@ def run_dab(args):
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-               "scaling": "weak", "vs_baseline": None, "dtype": "u32 popcount + f64 objective/rescale",
+               "scaling": "weak", "vs_baseline": None, "dtype": "u8 x u8 -> s32 tensor-core counts + f64 objective/rescale" if args.contraction == "tensor"
+               else "u32 popcount + f64 objective/rescale",
                "data": "synthetic", "config": workload_config(args), "clocks": clocks, "e2e": e2e,
                "gpu_launches": 3 * launches_per_kind,
                "kernel_ms_per_step": {k: v / args.steps for k, v in k_ms.items()},
                "binarize_gbs": binarize_gbs, "roofline": roofline, "roofline_contraction": roofline_contract,
-               "cpu_baseline": cpu_baseline}
+               "cpu_baseline": cpu_baseline, "contraction_wait_failures": dab.dab_contraction_wait_failures()}
         print(json.dumps(out))
     if world > 1:
         import torch.distributed as dist

@@ -18,8 +18,6 @@ namespace {
 
 constexpr int MMA_M = 128;       // activation rows per CTA = lanes of tensor memory
 constexpr int MMA_NMAX = 256;    // weight rows per CTA = columns of tensor memory
-constexpr int MMA_THREADS = 256;
-constexpr int MMA_STAGES = 2;
 constexpr long long kWaitCycles = 4000000000ll;  // about two seconds; a wait that long has failed
 
 __device__ unsigned int g_mma_wait_timeouts;
@@ -131,23 +129,33 @@ struct Side {
   int64_t rows;
 };
 
+// What the epilogue needs of one column-side row: its two values, its popcount K and n - K as doubles, and
+// its part of the output offset.
+struct __align__(16) ColumnParams {
+  double v1, v0, K, nK;
+  int64_t off;
+  int64_t pad;
+};
+
 // The pieces one thread expands per stage: unit u covers row (u>>3)/KQ*8 + (u&7), 16-byte piece (u>>3)%KQ.
 // Eight consecutive lanes hold the eight rows of one core matrix, so their 16-byte stores are one
 // contiguous 128 bytes; their loads read KQ x 16 contiguous bytes per row.
-constexpr int kMaxUnits = 3;
-
+//
+// One CTA forms one 128 x NT tile over the whole row length, 4*KQ mask words per stage.  There is a single
+// stage: a CTA alternates between expanding and waiting for the tensor cores, and the overlap comes from the
+// several CTAs resident on an SM (expansion, the fp64 rescale and the tensor pipe use different units), which
+// measured faster than two stages with fewer resident CTAs.
+//
 // kLanesAreActivations: the rows that ride the 128 lanes of tensor memory (and the threads of the epilogue)
 // are activation rows, the columns weight rows: coalesced stores when the output is contiguous along the
 // activation rows (NCHW).  Otherwise the roles are exchanged: coalesced for a row-major M x N output.
-template <int KQ, bool kLanesAreActivations>
-__global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const GemmArgs g) {
+template <int THREADS, int KQ, int MIN_CTAS, bool kLanesAreActivations>
+__global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(const GemmArgs g) {
   constexpr int KC = 8 * KQ;            // 16-byte K chunks per stage (two per mask word)
   constexpr uint32_t SBO = KC * 128;    // bytes between groups of 8 rows
-  extern __shared__ __align__(128) unsigned char stage_mem[];
-  __shared__ double s_v1[MMA_NMAX], s_v0[MMA_NMAX];  // column side
-  __shared__ int64_t s_off[MMA_NMAX];
-  __shared__ int s_K[MMA_NMAX];
-  __shared__ __align__(8) uint64_t s_bar[MMA_STAGES];
+  constexpr int kMaxUnits = ((MMA_M + MMA_NMAX) * KQ + THREADS - 1) / THREADS;
+  extern __shared__ __align__(128) unsigned char dyn_mem[];  // [lane-side stage][column-side stage][ColumnParams]
+  __shared__ __align__(8) uint64_t s_bar;
   __shared__ uint32_t s_tmem;
 
   const Side act{g.A, g.lda, g.KA, g.gamma, g.delta, g.M}, wgt{g.B, g.ldb, g.KB, g.alpha, g.beta, g.N};
@@ -164,9 +172,10 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
 
   const uint32_t a_bytes = MMA_M * KC * 16;
   const int ncap = (int)min((int64_t)MMA_NMAX, (S.rows + 15) & ~(int64_t)15);  // widest tile of this launch
-  const uint32_t stage_bytes = a_bytes + (uint32_t)ncap * KC * 16;
-  const uint32_t mem0 = (smem_u32(stage_mem) + 127u) & ~127u;
-  unsigned char* const mem0_ptr = stage_mem + (mem0 - smem_u32(stage_mem));
+  const uint32_t mem0 = (smem_u32(dyn_mem) + 127u) & ~127u;
+  unsigned char* const stage = dyn_mem + (mem0 - smem_u32(dyn_mem));
+  ColumnParams* const s_col = reinterpret_cast<ColumnParams*>(stage + a_bytes + (uint32_t)ncap * KC * 16);
+  const uint32_t bar = smem_u32(&s_bar);
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
@@ -175,20 +184,23 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid == 0) {
-#pragma unroll
-    for (int s = 0; s < MMA_STAGES; ++s) mbar_init(smem_u32(&s_bar[s]), 1);
+    mbar_init(bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // where activation row i and weight row j meet in the output: act_offset(i) + j * col_stride
   auto act_offset = [&](int64_t i) {
     return (i / g.map.inner) * g.map.outer_stride + (i % g.map.inner) * g.map.row_stride;
   };
-  for (int j = tid; j < MMA_NMAX; j += MMA_THREADS) {
-    const bool in = j < nrows;
-    s_v1[j] = in ? (double)S.v1[j0 + j] : 0.0;
-    s_v0[j] = in ? (double)S.v0[j0 + j] : 0.0;
-    s_K[j] = in ? S.K[j0 + j] : 0;
-    s_off[j] = !in ? 0 : kLanesAreActivations ? (j0 + j) * g.map.col_stride : act_offset(j0 + j);
+  for (int j = tid; j < nrows; j += THREADS) {
+    ColumnParams cp;
+    const int K = S.K[j0 + j];
+    cp.v1 = (double)S.v1[j0 + j];
+    cp.v0 = (double)S.v0[j0 + j];
+    cp.K = (double)K;
+    cp.nK = (double)(g.n - K);
+    cp.off = kLanesAreActivations ? (j0 + j) * g.map.col_stride : act_offset(j0 + j);
+    cp.pad = 0;
+    s_col[j] = cp;
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -199,13 +211,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
   // units of this thread: lane-side pieces first, then column-side pieces
   const int l_units = MMA_M * KQ, units = l_units + NT * KQ;
   const int chunks = (g.words + 4 * KQ - 1) / (4 * KQ);
+  const int real_words = (g.n + 31) >> 5;  // words beyond these hold no bits
   uint4 q[kMaxUnits];
 
   auto fetch = [&](int c) {  // the 16-byte pieces of chunk c, zero beyond the operands
     const int w0 = c * 4 * KQ;
 #pragma unroll
     for (int t = 0; t < kMaxUnits; ++t) {
-      const int u = tid + t * MMA_THREADS;
+      const int u = tid + t * THREADS;
       q[t] = make_uint4(0, 0, 0, 0);
       if (u >= units) continue;
       const bool isL = u < l_units;
@@ -222,22 +235,21 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
   };
 
   bool dead = false;
-  uint32_t parity[MMA_STAGES] = {0, 0};
+  uint32_t parity = 0;
   fetch(0);
   for (int c = 0; c < chunks; ++c) {
-    const int s = c & 1;
-    unsigned char* const stage = mem0_ptr + s * stage_bytes;
-    if (c >= MMA_STAGES) {  // the instructions that read this stage two chunks ago have completed
-      mbar_wait(smem_u32(&s_bar[s]), parity[s], dead);
-      parity[s] ^= 1;
+    if (c > 0) {  // the instructions that read the stage for the previous chunk have completed
+      mbar_wait(bar, parity, dead);
+      parity ^= 1;
     }
 #pragma unroll
     for (int t = 0; t < kMaxUnits; ++t) {
-      const int u = tid + t * MMA_THREADS;
+      const int u = tid + t * THREADS;
       if (u >= units) continue;
       const bool isL = u < l_units;
       const int v = isL ? u : u - l_units;
       const int group = (v >> 3) / KQ, piece = (v >> 3) % KQ;
+      if (c * 4 * KQ + 4 * piece >= g.words) continue;  // no instruction reads this part of the stage
       unsigned char* dst =
           stage + (isL ? 0u : a_bytes) + (uint32_t)group * SBO + (uint32_t)(8 * piece) * 128 + (v & 7) * 16;
       expand_words(q[t], dst);
@@ -247,34 +259,30 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
     __syncthreads();
     if (tid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t a_addr = mem0 + s * stage_bytes, b_addr = a_addr + a_bytes;
-      const int kw = min(4 * KQ, g.words - c * 4 * KQ);
+      const uint32_t a_addr = mem0, b_addr = mem0 + a_bytes;
+      const int kw = min(4 * KQ, real_words - c * 4 * KQ);
       for (int t = 0; t < kw; ++t)  // one mask word = 32 K bytes = two K chunks per instruction
         mma_i8(tmem, smem_desc(a_addr + t * 256, 128, SBO), smem_desc(b_addr + t * 256, 128, SBO), idesc,
                (c | t) != 0);
-      mma_commit(smem_u32(&s_bar[s]));
+      mma_commit(bar);
     }
   }
-  {  // the last commit covers every instruction issued before it
-    const int s = (chunks - 1) & 1;
-    mbar_wait(smem_u32(&s_bar[s]), parity[s], dead);
-  }
+  mbar_wait(bar, parity, dead);  // the last commit covers every instruction issued before it
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
   // Epilogue: thread = lane-side row (a warp reads the 32 lanes of its quarter), 32 columns at a time.
   {
     const int64_t gl = i0 + (warp & 3) * 32 + lane;
     const bool valid = gl < L.rows && !dead;
-    int Kl = 0;
-    double l1 = 0.0, l0 = 0.0;
+    double Kl = 0.0, l1 = 0.0, l0 = 0.0;
     int64_t off = 0;
     if (valid) {
-      Kl = L.K[gl];
+      Kl = (double)L.K[gl];
       l1 = (double)L.v1[gl];
       l0 = (double)L.v0[gl];
       off = kLanesAreActivations ? act_offset(gl) : gl * g.map.col_stride;
     }
-    for (int cb = warp >> 2; cb * 32 < NT; cb += 2) {
+    for (int cb = warp >> 2; cb * 32 < NT; cb += THREADS / 128) {
       uint32_t v[32];
       tmem_load_32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cb * 32), v);
       if (!valid) continue;
@@ -282,11 +290,24 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
       for (int jj = 0; jj < 32; ++jj) {
         const int j = cb * 32 + jj;
         if (j >= nrows) break;
-        const int p11 = (int)v[jj];
-        // rescale(p11, K of the weight row, K of the activation row, n, alpha, beta, gamma, delta)
-        g.C[off + s_off[j]] = kLanesAreActivations ? rescale(p11, s_K[j], Kl, g.n, s_v1[j], s_v0[j], l1, l0)
-                                                   : rescale(p11, Kl, s_K[j], g.n, l1, l0, s_v1[j], s_v0[j]);
-        if (g.p11) g.p11[kLanesAreActivations ? gl * g.ldp + j0 + j : (j0 + j) * g.ldp + gl] = p11;
+        const ColumnParams cp = s_col[j];
+        // The four counts as doubles (small integers: every difference is exact, so these are the values
+        // rescale() converts from int), then its four terms in its order: alpha gamma p11, alpha delta p10,
+        // beta gamma p01, beta delta p00, with p10 the count on the weight side only.
+        const double p11 = int_to_double((int)v[jj]);
+        const double pc = __dsub_rn(cp.K, p11), pl = __dsub_rn(Kl, p11);  // set on the column / lane side only
+        const double p00 = __dsub_rn(cp.nK, pl);
+        double y = __dmul_rn(__dmul_rn(cp.v1, l1), p11);
+        if (kLanesAreActivations) {
+          y = __dadd_rn(y, __dmul_rn(__dmul_rn(cp.v1, l0), pc));
+          y = __dadd_rn(y, __dmul_rn(__dmul_rn(cp.v0, l1), pl));
+        } else {
+          y = __dadd_rn(y, __dmul_rn(__dmul_rn(l1, cp.v0), pl));
+          y = __dadd_rn(y, __dmul_rn(__dmul_rn(l0, cp.v1), pc));
+        }
+        y = __dadd_rn(y, __dmul_rn(__dmul_rn(cp.v0, l0), p00));
+        g.C[off + cp.off] = (float)y;
+        if (g.p11) g.p11[kLanesAreActivations ? gl * g.ldp + j0 + j : (j0 + j) * g.ldp + gl] = (int)v[jj];
       }
     }
   }
@@ -296,22 +317,24 @@ __global__ void __launch_bounds__(MMA_THREADS, 2) binary_gemm_mma_kernel(const G
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
 }
 
-template <int KQ, bool kLanesAreActivations>
-cudaError_t launch_kq(const GemmArgs& args, dim3 grid, int ncap, cudaStream_t stream) {
-  const size_t smem_max = (size_t)MMA_STAGES * (MMA_M + MMA_NMAX) * (8 * KQ) * 16 + 128;
-  const size_t smem = (size_t)MMA_STAGES * (MMA_M + ncap) * (8 * KQ) * 16 + 128;
+inline size_t dynamic_bytes(int kq, int ncap) {
+  return (size_t)(MMA_M + ncap) * (8 * kq) * 16 + (size_t)ncap * sizeof(ColumnParams) + 128;
+}
+
+template <int THREADS, int KQ, int MIN_CTAS, bool kLanesAreActivations>
+cudaError_t launch_shape(const GemmArgs& args, dim3 grid, int ncap, cudaStream_t stream) {
   static bool configured[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  auto kernel = binary_gemm_mma_kernel<THREADS, KQ, MIN_CTAS, kLanesAreActivations>;
   if (!configured[dev]) {
-    e = cudaFuncSetAttribute(binary_gemm_mma_kernel<KQ, kLanesAreActivations>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynamic_bytes(KQ, MMA_NMAX));
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  binary_gemm_mma_kernel<KQ, kLanesAreActivations><<<grid, MMA_THREADS, smem, stream>>>(args);
+  kernel<<<grid, THREADS, dynamic_bytes(KQ, ncap), stream>>>(args);
   return cudaGetLastError();
 }
 
@@ -322,10 +345,12 @@ cudaError_t launch_side(const GemmArgs& args, cudaStream_t stream) {
   if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)gx, (unsigned)gy);
   const int ncap = (int)std::min<int64_t>(MMA_NMAX, (col_rows + 15) & ~(int64_t)15);
-  // Two CTAs per SM (so that one expands while the other's counts are rescaled) bound the stage size:
-  // eight mask words per stage for narrow column tiles, four otherwise.
-  return ncap <= 64 ? launch_kq<2, kLanesAreActivations>(args, grid, ncap, stream)
-                    : launch_kq<1, kLanesAreActivations>(args, grid, ncap, stream);
+  // CTA shape by tile width, from timings of the four layer shapes of the ResNet-18-like stack: narrow tiles
+  // run best as many small CTAs (six of 128 threads per SM), wider ones as fewer CTAs of 256 threads with
+  // longer stages (two per SM at the full 256 columns, where shared memory is the limit).
+  if (ncap <= 64) return launch_shape<128, 1, 6, kLanesAreActivations>(args, grid, ncap, stream);
+  if (ncap <= 128) return launch_shape<256, 1, 4, kLanesAreActivations>(args, grid, ncap, stream);
+  return launch_shape<256, 2, 2, kLanesAreActivations>(args, grid, ncap, stream);
 }
 
 }  // namespace

@@ -2,8 +2,9 @@
 
 `python -m paper_1804_02941_b200.sweep [--configs 1,2,3,4,5] [--batch5 256]` prints one JSON line per
 (config, layer or point, stage): device time by CUDA events (best of a few repetitions after warm-up), the
-stage's throughput and its fraction of the relevant roofline (HBM copy bandwidth for binarize and pack, the
-population-count rate for the contraction).  bench.py is the benchmark of record; this is the wider table.
+stage's throughput and its fraction of the relevant roofline (HBM copy bandwidth for binarize and pack; for the
+contraction, whichever kernel runs, alu_frac is its rate over the bound of the population-count kernel's
+instruction mix, so values above 1 are the tensor-core kernel beating the integer pipes).  bench.py is the benchmark of record; this is the wider table.
 """
 from __future__ import annotations
 
@@ -113,10 +114,13 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--batch5", type=int, default=256)
+    ap.add_argument("--contraction", default="tensor", choices=["tensor", "popc"])
     args = ap.parse_args()
+    dab.dab_set_contraction(dab.CONTRACT_TENSOR if args.contraction == "tensor" else dab.CONTRACT_POPC)
     want = set(args.configs.split(","))
     hbm, mhz, src = peaks()
     tops_peak = POPC_PER_CLK * WORDS_PER_POPC * SM_COUNT * mhz * 1e6 * 64 / 1e12
+    emit(contraction=args.contraction)
     emit(peaks=dict(hbm_gbs=hbm, source=src, contraction_tops_equiv=tops_peak,
                     contraction_peak="16 popc/clk/SM x 1.5 words/popc x 148 SMs x %.0f MHz x 64" % mhz))
     if "1" in want:
