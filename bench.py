@@ -48,8 +48,9 @@ def parse_args():
     ap.add_argument("--dense", action="store_true", help="N(0,1) inputs without zeros instead of post-ReLU inputs")
     ap.add_argument("--layers", default="", help="comma-separated layer names (e.g. l1_0,l4_1) to run a subset; "
                     "the default is the whole workload")
-    ap.add_argument("--contraction", default="tensor", choices=["tensor", "popc"],
-                    help="contraction kernel: tcgen05 tensor cores on byte-expanded masks (default) or AND + population counts")
+    ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"],
+                    help="contraction kernel: auto (tensor cores except on tiny problems; every layer of this workload takes "
+                         "them), tensor (forced) or popc (AND + population counts)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -238,7 +239,7 @@ def run_dab(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     dab.lib()
-    dab.dab_set_contraction(dab.CONTRACT_TENSOR if args.contraction == "tensor" else dab.CONTRACT_POPC)
+    dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
     hbm_peak, peak_src, sm_max_mhz = load_peaks()
 
     layers = select_layers(configs.config5(args.batch), args)
@@ -355,7 +356,7 @@ def run_dab(args):
     common = {"achieved": contract_tops, "unit": "TOPS-equiv", "avg_launch_ms": k_ms["contract"] / launches_per_kind,
               "share_of_step": k_ms["contract"] / sum(k_ms.values()), "output_store_gbs": store_gbs,
               "output_store_frac_of_hbm": store_gbs / hbm_peak}
-    if args.contraction == "tensor":
+    if args.contraction != "popc":
         int8_peak, int8_src = load_int8_peak()
         roofline_contract = {"kernel": "binary_gemm_mma_kernel", "bound": "tensor", "peak": int8_peak,
                              "frac": contract_tops / int8_peak, "peak_source": int8_src,
@@ -406,7 +407,7 @@ def run_dab(args):
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-               "scaling": "weak", "vs_baseline": None, "dtype": "u8 x u8 -> s32 tensor-core counts + f64 objective/rescale" if args.contraction == "tensor"
+               "scaling": "weak", "vs_baseline": None, "dtype": "u8 x u8 -> s32 tensor-core counts + f64 objective/rescale" if args.contraction != "popc"
                else "u32 popcount + f64 objective/rescale",
                "data": "synthetic", "config": workload_config(args), "clocks": clocks, "e2e": e2e,
                "gpu_launches": 3 * launches_per_kind,

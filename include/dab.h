@@ -215,13 +215,15 @@ dab_status dab_binary_conv_static(const dab_conv_desc* desc, const float* d_x, c
  * Which kernel forms the AND-popcounts of dab_binary_gemm and of every convolution entry point (Section 4.2
  * counts set bits with population-count instructions; an AND-popcount over n bits is also the dot product of
  * the two rows written as 0/1 bytes, which the tensor cores form exactly in 32-bit integers):
- *   DAB_CONTRACT_TENSOR  (default) mask words are expanded to bytes in shared memory and multiplied by
+ *   DAB_CONTRACT_TENSOR  mask words are expanded to bytes in shared memory and multiplied by
  *                        tcgen05.mma kind::i8 into tensor memory;
- *   DAB_CONTRACT_POPC    AND, carry-save adders and population counts on the integer pipes.
- * Both give the same counts bit for bit and apply the same four-term rescale.  The setting is process-wide and
- * read at each call; it exists so that the two can be measured against each other.
+ *   DAB_CONTRACT_POPC    AND, carry-save adders and population counts on the integer pipes;
+ *   DAB_CONTRACT_AUTO    (default) the tensor-core kernel, except for problems so small (fewer 128 x 64
+ *                        output tiles than the device has SMs) that its per-tile latency is all there is.
+ * Both kernels give the same counts and the same outputs bit for bit.  The setting is process-wide and read at
+ * each call; the two forced values exist so that the kernels can be tested and measured against each other.
  */
-typedef enum { DAB_CONTRACT_TENSOR = 0, DAB_CONTRACT_POPC = 1 } dab_contraction;
+typedef enum { DAB_CONTRACT_AUTO = 0, DAB_CONTRACT_TENSOR = 1, DAB_CONTRACT_POPC = 2 } dab_contraction;
 dab_status dab_set_contraction(dab_contraction path);
 dab_contraction dab_get_contraction(void);
 

@@ -326,11 +326,11 @@ def dab_popc_probe(blocks: int, iters: int, sink: torch.Tensor | None = None, st
     return sink
 
 
-CONTRACT_TENSOR, CONTRACT_POPC = 0, 1
+CONTRACT_AUTO, CONTRACT_TENSOR, CONTRACT_POPC = 0, 1, 2
 
 
 def dab_set_contraction(path: int) -> None:
-    """Process-wide choice of the contraction kernel: CONTRACT_TENSOR (default) or CONTRACT_POPC."""
+    """Process-wide choice of the contraction kernel: CONTRACT_AUTO (default), CONTRACT_TENSOR or CONTRACT_POPC."""
     _check(lib().dab_set_contraction(int(path)), "dab_set_contraction")
 
 

@@ -15,16 +15,18 @@ inline dab_status from_cuda(cudaError_t e) { return e == cudaSuccess ? DAB_OK : 
 
 constexpr size_t kAlign = 256;
 
-std::atomic<int> g_contraction{(int)DAB_CONTRACT_TENSOR};
+std::atomic<int> g_contraction{(int)DAB_CONTRACT_AUTO};
 
 // The contraction kernel the process-wide setting names.  The tensor-core kernel tiles the column side
-// (weights when lanes_along_rows, activations otherwise) 256 rows per grid row; a launch too tall for
-// that takes the population-count kernel.
+// (weights when lanes_along_rows, activations otherwise) at least 64 rows per grid row; a launch too tall for
+// that takes the population-count kernel, and so does, under DAB_CONTRACT_AUTO, one with fewer 128 x 64 tiles
+// than a B200 has SMs: there the tensor-core kernel is a chain of dependent stage rounds on a few SMs.
 cudaError_t contract(const GemmArgs& g, bool lanes_along_rows, cudaStream_t stream) {
-  const int64_t column_rows = lanes_along_rows ? g.N : g.M;
-  if (g_contraction.load(std::memory_order_relaxed) == (int)DAB_CONTRACT_TENSOR && column_rows <= (int64_t)65535 * 256)
-    return launch_gemm_mma(g, lanes_along_rows, stream);
-  return launch_gemm(g, lanes_along_rows, stream);
+  const int64_t lane_rows = lanes_along_rows ? g.M : g.N, column_rows = lanes_along_rows ? g.N : g.M;
+  const int mode = g_contraction.load(std::memory_order_relaxed);
+  bool tensor = mode != (int)DAB_CONTRACT_POPC && column_rows <= (int64_t)65535 * 64;
+  if (mode == (int)DAB_CONTRACT_AUTO && ((lane_rows + 127) / 128) * ((column_rows + 63) / 64) < 148) tensor = false;
+  return tensor ? launch_gemm_mma(g, lanes_along_rows, stream) : launch_gemm(g, lanes_along_rows, stream);
 }
 
 struct ConvGeom {
@@ -368,7 +370,7 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
 }
 
 dab_status dab_set_contraction(dab_contraction path) {
-  if (path != DAB_CONTRACT_TENSOR && path != DAB_CONTRACT_POPC) return DAB_ERR_INVALID_ARG;
+  if (path != DAB_CONTRACT_AUTO && path != DAB_CONTRACT_TENSOR && path != DAB_CONTRACT_POPC) return DAB_ERR_INVALID_ARG;
   g_contraction.store((int)path, std::memory_order_relaxed);
   return DAB_OK;
 }

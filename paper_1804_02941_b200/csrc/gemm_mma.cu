@@ -149,11 +149,11 @@ struct __align__(16) ColumnParams {
 // kLanesAreActivations: the rows that ride the 128 lanes of tensor memory (and the threads of the epilogue)
 // are activation rows, the columns weight rows: coalesced stores when the output is contiguous along the
 // activation rows (NCHW).  Otherwise the roles are exchanged: coalesced for a row-major M x N output.
-template <int THREADS, int KQ, int MIN_CTAS, bool kLanesAreActivations>
-__global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(const GemmArgs g) {
+template <int THREADS, int KQ, int MIN_CTAS, int NT_MAX, bool kLanesAreActivations>
+__global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(const GemmArgs g, const int tile_cols) {
   constexpr int KC = 8 * KQ;            // 16-byte K chunks per stage (two per mask word)
   constexpr uint32_t SBO = KC * 128;    // bytes between groups of 8 rows
-  constexpr int kMaxUnits = ((MMA_M + MMA_NMAX) * KQ + THREADS - 1) / THREADS;
+  constexpr int kMaxUnits = ((MMA_M + NT_MAX) * KQ + THREADS - 1) / THREADS;  // NT <= NT_MAX in this shape
   extern __shared__ __align__(128) unsigned char dyn_mem[];  // [lane-side stage][column-side stage][ColumnParams]
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ uint32_t s_tmem;
@@ -164,14 +164,14 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int64_t i0 = (int64_t)blockIdx.x * MMA_M;
-  const int64_t j0 = (int64_t)blockIdx.y * MMA_NMAX;
-  const int nrows = (int)min((int64_t)MMA_NMAX, S.rows - j0);  // column-side rows of this tile
+  const int64_t j0 = (int64_t)blockIdx.y * tile_cols;        // tile_cols: 64, 128 or 256 column-side rows per CTA
+  const int nrows = (int)min((int64_t)tile_cols, S.rows - j0);  // column-side rows of this tile
   const int NT = (nrows + 15) & ~15;                            // instruction N
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < NT) tmem_cols <<= 1;
 
   const uint32_t a_bytes = MMA_M * KC * 16;
-  const int ncap = (int)min((int64_t)MMA_NMAX, (S.rows + 15) & ~(int64_t)15);  // widest tile of this launch
+  const int ncap = (int)min((int64_t)tile_cols, (S.rows + 15) & ~(int64_t)15);  // widest tile of this launch
   const uint32_t mem0 = (smem_u32(dyn_mem) + 127u) & ~127u;
   unsigned char* const stage = dyn_mem + (mem0 - smem_u32(dyn_mem));
   ColumnParams* const s_col = reinterpret_cast<ColumnParams*>(stage + a_bytes + (uint32_t)ncap * KC * 16);
@@ -321,36 +321,40 @@ inline size_t dynamic_bytes(int kq, int ncap) {
   return (size_t)(MMA_M + ncap) * (8 * kq) * 16 + (size_t)ncap * sizeof(ColumnParams) + 128;
 }
 
-template <int THREADS, int KQ, int MIN_CTAS, bool kLanesAreActivations>
-cudaError_t launch_shape(const GemmArgs& args, dim3 grid, int ncap, cudaStream_t stream) {
+template <int THREADS, int KQ, int MIN_CTAS, int NT_MAX, bool kLanesAreActivations>
+cudaError_t launch_shape(const GemmArgs& args, dim3 grid, int tile_cols, int ncap, cudaStream_t stream) {
   static bool configured[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  auto kernel = binary_gemm_mma_kernel<THREADS, KQ, MIN_CTAS, kLanesAreActivations>;
+  auto kernel = binary_gemm_mma_kernel<THREADS, KQ, MIN_CTAS, NT_MAX, kLanesAreActivations>;
   if (!configured[dev]) {
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynamic_bytes(KQ, MMA_NMAX));
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynamic_bytes(KQ, NT_MAX));
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  kernel<<<grid, THREADS, dynamic_bytes(KQ, ncap), stream>>>(args);
+  kernel<<<grid, THREADS, dynamic_bytes(KQ, ncap), stream>>>(args, tile_cols);
   return cudaGetLastError();
 }
 
 template <bool kLanesAreActivations>
 cudaError_t launch_side(const GemmArgs& args, cudaStream_t stream) {
   const int64_t lane_rows = kLanesAreActivations ? args.M : args.N, col_rows = kLanesAreActivations ? args.N : args.M;
-  const int64_t gx = (lane_rows + MMA_M - 1) / MMA_M, gy = (col_rows + MMA_NMAX - 1) / MMA_NMAX;
+  // Column tile: the full 256 columns of an accumulator unless that leaves most SMs without a CTA.
+  const int64_t gx = (lane_rows + MMA_M - 1) / MMA_M;
+  int tile_cols = MMA_NMAX;
+  while (tile_cols > 64 && gx * ((col_rows + tile_cols - 1) / tile_cols) < 2 * 148) tile_cols >>= 1;
+  const int64_t gy = (col_rows + tile_cols - 1) / tile_cols;
   if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)gx, (unsigned)gy);
-  const int ncap = (int)std::min<int64_t>(MMA_NMAX, (col_rows + 15) & ~(int64_t)15);
+  const int ncap = (int)std::min<int64_t>(tile_cols, (col_rows + 15) & ~(int64_t)15);
   // CTA shape by tile width, from timings of the four layer shapes of the ResNet-18-like stack: narrow tiles
   // run best as many small CTAs (six of 128 threads per SM), wider ones as fewer CTAs of 256 threads with
   // longer stages (two per SM at the full 256 columns, where shared memory is the limit).
-  if (ncap <= 64) return launch_shape<128, 1, 6, kLanesAreActivations>(args, grid, ncap, stream);
-  if (ncap <= 128) return launch_shape<256, 1, 4, kLanesAreActivations>(args, grid, ncap, stream);
-  return launch_shape<256, 2, 2, kLanesAreActivations>(args, grid, ncap, stream);
+  if (ncap <= 64) return launch_shape<128, 1, 6, 64, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
+  if (ncap <= 128) return launch_shape<256, 1, 4, 128, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
+  return launch_shape<256, 2, 2, MMA_NMAX, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
 }
 
 }  // namespace

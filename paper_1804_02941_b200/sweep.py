@@ -114,9 +114,9 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--batch5", type=int, default=256)
-    ap.add_argument("--contraction", default="tensor", choices=["tensor", "popc"])
+    ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"])
     args = ap.parse_args()
-    dab.dab_set_contraction(dab.CONTRACT_TENSOR if args.contraction == "tensor" else dab.CONTRACT_POPC)
+    dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
     want = set(args.configs.split(","))
     hbm, mhz, src = peaks()
     tops_peak = POPC_PER_CLK * WORDS_PER_POPC * SM_COUNT * mhz * 1e6 * 64 / 1e12

@@ -1,4 +1,4 @@
-"""GPU parity of the two contraction kernels: tensor cores (default) and population counts.
+"""GPU parity of the two contraction kernels, each forced: tensor cores and population counts.
 
 Both must give the checker's AND-popcounts bit for bit, outputs within 1e-5 relative, and, because they share
 the rescale arithmetic, outputs identical to each other.  Shapes cover one and several column tiles (256
@@ -22,7 +22,7 @@ def dab():
     d.lib()
     oracle.set_threads(8)
     yield d
-    d.dab_set_contraction(d.CONTRACT_TENSOR)
+    d.dab_set_contraction(d.CONTRACT_AUTO)
 
 
 @contextlib.contextmanager
@@ -35,14 +35,15 @@ def contraction(dab, path):
         dab.dab_set_contraction(before)
 
 
-def test_default_is_the_tensor_core_kernel_and_setter_validates(dab):
-    assert dab.dab_get_contraction() == dab.CONTRACT_TENSOR
-    with contraction(dab, dab.CONTRACT_POPC):
-        assert dab.dab_get_contraction() == dab.CONTRACT_POPC
-    assert dab.dab_get_contraction() == dab.CONTRACT_TENSOR
+def test_default_is_automatic_and_setter_validates(dab):
+    assert dab.dab_get_contraction() == dab.CONTRACT_AUTO
+    for path in (dab.CONTRACT_POPC, dab.CONTRACT_TENSOR):
+        with contraction(dab, path):
+            assert dab.dab_get_contraction() == path
+    assert dab.dab_get_contraction() == dab.CONTRACT_AUTO
     with pytest.raises(dab.DabError):
         dab.dab_set_contraction(7)
-    assert dab.dab_get_contraction() == dab.CONTRACT_TENSOR
+    assert dab.dab_get_contraction() == dab.CONTRACT_AUTO
 
 
 GEMM_SHAPES = [(1, 1, 1), (3, 2, 31), (128, 16, 32), (129, 17, 33), (300, 80, 576), (130, 64, 1152), (257, 300, 4608),
