@@ -175,6 +175,24 @@ def conv(x, w_e, w_alpha, w_beta, kh, kw, stride=(1, 1), pad=(0, 0), details=Tru
     return ConvResult(y, p_e, p_K, p_g, p_d, p_f, p_p)
 
 
+def conv_wbin(x, w_e, w_alpha, w_beta, kh, kw, stride=(1, 1), pad=(0, 0)):
+    """I (*) W~ with fp32 activations and two-level filters (Section 4.3.2, weights-only binarization).
+    Returns (y fp32, abs_terms fp64), both N x Cout x Ho x Wo."""
+    x = np.ascontiguousarray(x, np.float32)
+    w_e = np.ascontiguousarray(w_e, np.uint8)
+    w_alpha = np.ascontiguousarray(w_alpha, np.float32)
+    w_beta = np.ascontiguousarray(w_beta, np.float32)
+    N, Cc, H, W = x.shape
+    Cout, n = w_e.shape
+    assert n == Cc * kh * kw
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    d = _desc(x.shape, Cout, kh, kw, stride, pad)
+    y = np.zeros((N, Cout, Ho, Wo), np.float32)
+    mag = np.zeros((N, Cout, Ho, Wo), np.float64)
+    lib().oracle_conv_wbin(C.byref(d), _p(x), _p(w_e), _p(w_alpha), _p(w_beta), _p(y), _p(mag))
+    return y, mag
+
+
 def im2col(x, kh, kw, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     """Patch rows (N*Ho*Wo) x (C*kh*kw), element order (c, kh, kw), zero padding as 0.0 values."""
     x = np.ascontiguousarray(x, np.float32)

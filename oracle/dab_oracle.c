@@ -288,3 +288,39 @@ void oracle_conv_sign(const oracle_conv_desc* d, const float* x, const uint8_t* 
                       uint32_t* p_flags, int32_t* p_p11) {
   conv_with_coder(1, d, x, w_e, w_alpha, w_beta, y, p_e, p_K, p_gamma, p_delta, p_flags, p_p11);
 }
+
+/* Section 4.3.2, weights-only binarization: the plain convolution of the fp32 input with the two-level
+ * filters W~ = alpha*e + beta*(1-e).  Every product and the running sum are fp64, in element order
+ * (c, kh, kw); one rounding to fp32 at the end. */
+void oracle_conv_wbin(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
+                      const float* w_beta, float* y, double* abs_terms) {
+  int32_t Ho, Wo;
+  int32_t n = d->C * d->kh * d->kw;
+  int64_t patches, pi;
+  conv_out_size(d, &Ho, &Wo);
+  patches = (int64_t)d->N * Ho * Wo;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
+#endif
+  for (pi = 0; pi < patches; ++pi) {
+    int32_t img = (int32_t)(pi / ((int64_t)Ho * Wo));
+    int32_t ho = (int32_t)((pi / Wo) % Ho);
+    int32_t wo = (int32_t)(pi % Wo);
+    float* p = (float*)malloc(sizeof(float) * (size_t)n);
+    int32_t co, i;
+    extract_patch(d, x, img, ho, wo, p);
+    for (co = 0; co < d->Cout; ++co) {
+      const uint8_t* e = w_e + (int64_t)co * n;
+      double a = (double)w_alpha[co], b = (double)w_beta[co], acc = 0.0, mag = 0.0;
+      int64_t o = (((int64_t)img * d->Cout + co) * Ho + ho) * Wo + wo;
+      for (i = 0; i < n; ++i) {
+        double t = (double)p[i] * (e[i] ? a : b);
+        acc = acc + t;
+        mag = mag + fabs(t);
+      }
+      y[o] = (float)acc;
+      if (abs_terms) abs_terms[o] = mag;
+    }
+    free(p);
+  }
+}

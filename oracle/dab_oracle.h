@@ -95,6 +95,17 @@ void oracle_conv_sign(const oracle_conv_desc* d, const float* x, const uint8_t* 
                       const float* w_beta, float* y, uint8_t* p_e, int32_t* p_K, float* p_gamma, float* p_delta,
                       uint32_t* p_flags, int32_t* p_p11);
 
+/*
+ * Section 4.3.2 forward pass with weights-only binarization (the paper's WBin networks): the fp32 input is
+ * convolved with the two-level filters W~ = alpha*e + beta*(1-e); nothing is done to the activations.
+ *   y[img][co][ho][wo] = sum over (c, kh, kw) of x_patch[i] * (e_co[i] ? alpha_co : beta_co)
+ * Products and the running sum are fp64, elements taken in (c, kh, kw) order, one rounding to fp32.
+ * abs_terms (nullable, same shape as y, fp64) receives the sum of |product|: the scale rounding errors of any
+ * other summation order are measured against.
+ */
+void oracle_conv_wbin(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
+                      const float* w_beta, float* y, double* abs_terms);
+
 /* Patch extraction alone (explicit loops), rows = N*Ho*Wo, row length C*kh*kw. */
 void oracle_im2col(const oracle_conv_desc* d, const float* x, float* patches);
 
