@@ -172,6 +172,24 @@ dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, con
                                 void* stream);
 
 /*
+ * dab_wbin_conv — Section 4.3.2 / Corollary 1 as the paper's weights-only ("WBin") networks run it: the
+ * full-precision input convolved with the two-level filters W~ = alpha e + beta (1 - e),
+ *   y[img][co][ho][wo] = alpha_co * (sum of the patch values under e_co) + beta_co * (sum of the others),
+ * with nothing done to the activations.  Patch definition, element order (c, kh, kw), zero padding and output
+ * layout as in dab_binary_conv; the filters come from dab_binarize on the [Cout x C*kh*kw] weight matrix
+ * (their K is not needed).  No workspace.
+ *
+ * Arithmetic: each patch is taken as 32-bit fixed point relative to its own largest magnitude and the sums
+ * under e are formed exactly in integers on the tensor cores, so the result differs from exact arithmetic by
+ * at most 2^-32 * n * max|x_patch| * max(|alpha|, |beta|) plus the final rounding to fp32 (patches whose largest
+ * magnitude is subnormal are resolved to 2^-158 instead).  A patch that contains a NaN or an infinity gives NaN
+ * in all its outputs.  C*H*W must be below 2^31.
+ * DAB_ERR_UNSUPPORTED if no tile of the layer fits shared memory (kernels wider than about 200 columns).
+ */
+dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                         const float* d_walpha, const float* d_wbeta, float* d_y, void* stream);
+
+/*
  * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up
  * to 16 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
  * chunks overlap on three streams, and the call returns after everything has drained.  Use pinned host memory:

@@ -24,7 +24,7 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
-           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures")
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv")
 
 
 class DabError(RuntimeError):
@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_static_capacity.argtypes = []
         L.dab_binary_conv_static.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
+        L.dab_wbin_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
         L.dab_set_contraction.argtypes = [i32]
         L.dab_get_contraction.argtypes = []
         L.dab_contraction_wait_failures.argtypes = [vp]
@@ -316,6 +317,23 @@ def dab_binary_conv_static(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(
     st = lib().dab_binary_conv_static(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha),
                                       _ptr(w.beta), _ptr(y), _stream(stream))
     _check(st, "dab_binary_conv_static")
+    return y
+
+
+def dab_wbin_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
+                  y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Weights-only binarized convolution: fp32 NCHW input against the two-level filters `w` (no workspace)."""
+    _dev(x, torch.float32, "x")
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous NCHW")
+    Cout = w.mask.shape[0]
+    desc = make_desc(tuple(x.shape), Cout, kh, kw, stride, pad)
+    Ho, Wo = dab_conv_output_size(desc)
+    if y is None:
+        y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=x.device)
+    st = lib().dab_wbin_conv(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.alpha), _ptr(w.beta), _ptr(y),
+                             _stream(stream))
+    _check(st, "dab_wbin_conv")
     return y
 
 

@@ -379,9 +379,26 @@ dab_contraction dab_get_contraction(void) { return (dab_contraction)g_contractio
 
 dab_status dab_contraction_wait_failures(uint32_t* h_count) {
   if (!h_count) return DAB_ERR_INVALID_ARG;
-  unsigned int c = 0;
+  unsigned int c = 0, w = 0;
   cudaError_t e = read_mma_wait_timeouts(&c);
-  *h_count = c;
+  if (e == cudaSuccess) e = read_wbin_wait_timeouts(&w);
+  *h_count = c + w;
+  return from_cuda(e);
+}
+
+dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
+                         const float* d_walpha, const float* d_wbeta, float* d_y, void* stream) {
+  if (!desc) return DAB_ERR_INVALID_ARG;
+  if (desc->C > 0 && desc->kh > 0 && desc->kw > 0 && (int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N)
+    return DAB_ERR_UNSUPPORTED;
+  ConvGeom g;
+  if (!conv_geom(desc, &g)) return DAB_ERR_INVALID_ARG;
+  if (!d_x || !d_wmask || !d_walpha || !d_wbeta || !d_y) return DAB_ERR_INVALID_ARG;
+  if (ldw < dab_words_per_row(g.n) || (ldw & 3) || !aligned16(d_wmask)) return DAB_ERR_INVALID_ARG;
+  if (desc->Cout > 65535 * 64 || (int64_t)desc->C * desc->H * desc->W > 0x7FFFFFFF) return DAB_ERR_UNSUPPORTED;
+  cudaError_t e = launch_wbin_conv(*desc, g.Ho, g.Wo, d_x, d_wmask, ldw, d_walpha, d_wbeta, d_y,
+                                   static_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return DAB_ERR_UNSUPPORTED;  // no tile of this layer fits shared memory
   return from_cuda(e);
 }
 

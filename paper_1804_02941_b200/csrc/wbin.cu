@@ -1,0 +1,349 @@
+// Weights-only binarized convolution (Section 4.3.2, Corollary 1: the forward pass I (*) W~ with
+// W~ = alpha e + beta (1 - e) and full-precision activations), on the tensor cores.
+//
+//   y[p][co] = alpha_co * M1 + beta_co * (S - M1),   M1 = sum_{i: e_co[i] = 1} x_p[i],   S = sum_i x_p[i]
+//
+// M1 is a dense contraction of the patch matrix with the 0/1 filter masks.  It is formed exactly in integers:
+// every patch row is written as 32-bit fixed point relative to its own largest magnitude
+// (q_i = rint(x_i * 2^sexp), |q_i| < 2^31), q is split into its four bytes (three unsigned, the top one
+// signed), and four tcgen05.mma kind::i8 products with the masks expanded to 0/1 bytes give four 32-bit
+// accumulators per output in tensor memory; M1 = a3 2^24 + a2 2^16 + a1 2^8 + a0 (times 2^-sexp).  The only
+// error is the rounding of x_i to q_i: at most 2^-32 of the row's largest magnitude per element.
+//
+// A CTA owns a tile of TH x TW output positions of one image (at most 128 = the lanes of tensor memory) and 64
+// filters.  It never forms patches in global memory: for each group of 128 patch elements it stages the
+// channels they come from in shared memory, and every thread gathers 16 consecutive elements of its row,
+// converts them and stores one 16-byte K chunk per byte plane in the operand layout of tc.cuh.
+#include <algorithm>
+#include <climits>
+
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace dab {
+namespace {
+
+using namespace tc;
+
+__device__ unsigned int g_wbin_wait_timeouts;
+
+constexpr int WB_THREADS = 256;
+constexpr int WB_JS = 4;                         // mask words (k-steps of 32 elements) per stage
+constexpr int WB_KS = WB_JS * 32;                // patch elements per stage
+constexpr int WB_KC = WB_JS * 2;                 // 16-byte K chunks per stage
+constexpr int WB_NT = 64;                        // filters per CTA
+constexpr uint32_t WB_SBO = WB_KC * 128;         // bytes between groups of 8 rows
+constexpr uint32_t WB_PLANE = kLanes * WB_KS;    // bytes of one byte plane of the activation stage
+constexpr uint32_t WB_BSTAGE = WB_NT * WB_KS;    // bytes of the filter stage
+constexpr uint16_t kNoElement = 0xFFFFu;
+
+struct WbinArgs {
+  dab_conv_desc d;
+  int32_t Ho, Wo, n, words, khw;
+  int32_t TH, TW, tiles_h, tiles_w;
+  int32_t in_h, in_w, pitch, ch_words, max_ch;
+  uint32_t magic_npix, magic_in_w, magic_khw, magic_kw;  // ceil(2^32 / d): floor(i / d) = umulhi(i, magic); 0 if d == 1
+  const float* x;
+  const uint32_t* wmask;
+  int32_t ldw;
+  const float* walpha;
+  const float* wbeta;
+  float* y;
+};
+
+__device__ __forceinline__ int fast_div(int i, uint32_t magic) {
+  return magic ? (int)__umulhi((unsigned)i, magic) : i;
+}
+
+// Byte planes of four fixed-point values: out[p] holds byte p of q0..q3 (q0 in the lowest byte).
+__device__ __forceinline__ void byte_planes(uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3, uint32_t (&out)[4]) {
+  const uint32_t a = __byte_perm(q0, q1, 0x5140), b = __byte_perm(q0, q1, 0x7362);
+  const uint32_t c = __byte_perm(q2, q3, 0x5140), d = __byte_perm(q2, q3, 0x7362);
+  out[0] = __byte_perm(a, c, 0x5410);
+  out[1] = __byte_perm(a, c, 0x7632);
+  out[2] = __byte_perm(b, d, 0x5410);
+  out[3] = __byte_perm(b, d, 0x7632);
+}
+
+__global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs a) {
+  extern __shared__ __align__(128) unsigned char dyn_mem[];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_rowsexp[kLanes];      // scale exponent of a row; INT_MIN: row not in the image; INT_MAX: non-finite
+  __shared__ int s_rowsum[2][kLanes][4]; // byte-plane sums of q over the row, one set per gathering thread
+  __shared__ double s_alpha[WB_NT], s_beta[WB_NT];
+  __shared__ uint16_t s_off[WB_KS];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t mem0 = (smem_u32(dyn_mem) + 127u) & ~127u;
+  unsigned char* const stage_a = dyn_mem + (mem0 - smem_u32(dyn_mem));
+  unsigned char* const stage_b = stage_a + 4 * WB_PLANE;
+  float* const tile = reinterpret_cast<float*>(stage_b + WB_BSTAGE);
+  uint32_t* const pixmax = reinterpret_cast<uint32_t*>(tile + (size_t)a.max_ch * a.ch_words);
+  const uint32_t bar = smem_u32(&s_bar);
+
+  // tile of this CTA
+  const int tiles_per_img = a.tiles_h * a.tiles_w;
+  const int img = blockIdx.x / tiles_per_img, trem = blockIdx.x % tiles_per_img;
+  const int ho0 = (trem / a.tiles_w) * a.TH, wo0 = (trem % a.tiles_w) * a.TW;
+  const int h0 = ho0 * a.d.stride_h - a.d.pad_h, w0 = wo0 * a.d.stride_w - a.d.pad_w;
+  const int j0 = blockIdx.y * WB_NT;
+  const float* const ximg = a.x + (int64_t)img * a.d.C * a.d.H * a.d.W;
+  const int npix = a.in_h * a.in_w;
+
+  if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 4 * WB_NT);
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int j = tid; j < WB_NT; j += WB_THREADS) {
+    const bool in = j0 + j < a.d.Cout;
+    s_alpha[j] = in ? (double)a.walpha[j0 + j] : 0.0;
+    s_beta[j] = in ? (double)a.wbeta[j0 + j] : 0.0;
+  }
+  for (int p = tid; p < npix; p += WB_THREADS) pixmax[p] = 0u;
+  __syncthreads();
+
+  // Largest magnitude over the channels of every staged pixel (as bit patterns: NaN > Inf > finite).
+  for (int idx = tid; idx < a.d.C * npix; idx += WB_THREADS) {
+    const int c = fast_div(idx, a.magic_npix), pix = idx - c * npix;
+    const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
+    const int h = h0 + r, w = w0 + s;
+    if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W) {
+      const uint32_t m = __float_as_uint(__ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w)) & 0x7FFFFFFFu;
+      if (m) atomicMax(&pixmax[pix], m);
+    }
+  }
+  __syncthreads();
+
+  // Row = output position (lh, lw) of the tile; its scale comes from the largest magnitude of its patch.
+  const int row = tid & (kLanes - 1), half = tid >> 7;
+  const int lh = row / a.TW, lw = row - lh * a.TW;
+  const bool row_in = lh < a.TH && ho0 + lh < a.Ho && wo0 + lw < a.Wo;
+  const int origin = lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+  if (tid < kLanes) {
+    int sexp = INT_MIN;
+    if (row_in) {
+      uint32_t m = 0u;
+      for (int i = 0; i < a.d.kh; ++i)
+        for (int j = 0; j < a.d.kw; ++j)
+          m = max(m, pixmax[(lh * a.d.stride_h + i) * a.in_w + lw * a.d.stride_w + j]);
+      if (m >= 0x7F800000u) sexp = INT_MAX;
+      else if (m == 0u) sexp = 0;
+      else sexp = 30 - ((int)(m >> 23) - 127);  // -97 .. 157 (the largest for a subnormal maximum)
+    }
+    s_rowsexp[row] = sexp;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+  const int my_sexp = s_rowsexp[row];
+  const bool gather = row_in && my_sexp != INT_MAX;
+  // x * 2^sexp in two exact steps: 2^sexp itself is beyond fp32 for the smallest patches
+  const int sexp1 = gather ? min(my_sexp, 100) : 0, sexp2 = gather ? my_sexp - sexp1 : 0;
+  const float fac = __int_as_float((sexp1 + 127) << 23), fac2 = __int_as_float((sexp2 + 127) << 23);
+  const uint32_t idesc_u = instr_desc(WB_NT, false), idesc_s = instr_desc(WB_NT, true);
+
+  int psum[4] = {0, 0, 0, 0};
+  bool dead = false;
+  uint32_t parity = 0;
+  const int stages = (a.words + WB_JS - 1) / WB_JS;
+  for (int st = 0; st < stages; ++st) {
+    const int k0 = st * WB_KS;
+    const int k1 = min(a.n, k0 + WB_KS);
+    const int c_lo = fast_div(k0, a.magic_khw), c_hi = fast_div(k1 - 1, a.magic_khw) + 1;
+    // (1) stage the channels this group of elements comes from; offsets of the elements inside the staged tile
+    for (int idx = tid; idx < (c_hi - c_lo) * npix; idx += WB_THREADS) {
+      const int c = fast_div(idx, a.magic_npix), pix = idx - c * npix;
+      const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
+      const int h = h0 + r, w = w0 + s;
+      float v = 0.0f;
+      if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
+        v = __ldg(ximg + ((int64_t)(c_lo + c) * a.d.H + h) * a.d.W + w);
+      tile[c * a.ch_words + r * a.pitch + s] = v;
+    }
+    if (tid < WB_KS) {
+      const int k = k0 + tid;
+      uint16_t o = kNoElement;
+      if (k < a.n) {
+        const int c = fast_div(k, a.magic_khw), rs = k - c * a.khw;
+        const int r = fast_div(rs, a.magic_kw), s = rs - r * a.d.kw;
+        o = (uint16_t)((c - c_lo) * a.ch_words + r * a.pitch + s);
+      }
+      s_off[tid] = o;
+    }
+    __syncthreads();
+    // (2) the tensor cores have finished reading the previous contents of the operand stages
+    if (st > 0) {
+      mbar_wait(bar, parity, dead, &g_wbin_wait_timeouts);
+      parity ^= 1;
+    }
+    // (3) gather, convert, split into byte planes: thread = (row, every other 16-element chunk)
+    if (gather) {
+      const float* const src = tile + origin;
+#pragma unroll
+      for (int t = 0; t < WB_KC / 2; ++t) {
+        const int kc = half + 2 * t;
+        if (k0 + kc * 16 >= a.n) break;
+        uint32_t pl[4][4];
+#pragma unroll
+        for (int g4 = 0; g4 < 4; ++g4) {
+          uint32_t q[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const uint16_t o = s_off[kc * 16 + g4 * 4 + e];
+            const float v = (o != kNoElement) ? src[o] : 0.0f;
+            q[e] = (uint32_t)__float2int_rn(__fmul_rn(__fmul_rn(v, fac), fac2));
+          }
+          uint32_t w4[4];
+          byte_planes(q[0], q[1], q[2], q[3], w4);
+#pragma unroll
+          for (int p = 0; p < 4; ++p) pl[p][g4] = w4[p];
+          psum[0] = (int)__dp4a(w4[0], 0x01010101u, (unsigned)psum[0]);
+          psum[1] = (int)__dp4a(w4[1], 0x01010101u, (unsigned)psum[1]);
+          psum[2] = (int)__dp4a(w4[2], 0x01010101u, (unsigned)psum[2]);
+          psum[3] = __dp4a((int)w4[3], 0x01010101, psum[3]);
+        }
+        unsigned char* dst = stage_a + (uint32_t)(row >> 3) * WB_SBO + (uint32_t)kc * 128 + (row & 7) * 16;
+#pragma unroll
+        for (int p = 0; p < 4; ++p)
+          *reinterpret_cast<uint4*>(dst + p * WB_PLANE) = make_uint4(pl[p][0], pl[p][1], pl[p][2], pl[p][3]);
+      }
+    }
+    // (4) the masks of the 64 filters: four words of a row -> eight K chunks of 0/1 bytes
+    if (tid < WB_NT) {
+      uint4 q = make_uint4(0, 0, 0, 0);
+      const int w0m = st * WB_JS;
+      if (j0 + tid < a.d.Cout && w0m < a.ldw)
+        q = *reinterpret_cast<const uint4*>(a.wmask + (int64_t)(j0 + tid) * a.ldw + w0m);
+      expand_words(q, stage_b + (uint32_t)(tid >> 3) * WB_SBO + (tid & 7) * 16);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> tensor-core reads
+    __syncthreads();
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t b_addr = mem0 + 4 * WB_PLANE;
+      const int kw = min(WB_JS, a.words - st * WB_JS);
+      for (int t = 0; t < kw; ++t) {
+        const uint64_t db = smem_desc(b_addr + t * 256, 128, WB_SBO);
+        for (int p = 0; p < 4; ++p)
+          mma_i8(tmem + (uint32_t)(p * WB_NT), smem_desc(mem0 + p * WB_PLANE + t * 256, 128, WB_SBO), db,
+                 p == 3 ? idesc_s : idesc_u, (st | t) != 0);
+      }
+      mma_commit(bar);
+    }
+  }
+  s_rowsum[half][row][0] = psum[0];
+  s_rowsum[half][row][1] = psum[1];
+  s_rowsum[half][row][2] = psum[2];
+  s_rowsum[half][row][3] = psum[3];
+  mbar_wait(bar, parity, dead, &g_wbin_wait_timeouts);  // the last commit covers every instruction before it
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  __syncthreads();
+
+  // Epilogue: thread = row (a warp reads the 32 lanes of its quarter), warps 0-3 the first 32 filters, 4-7 the rest.
+  {
+    const int erow = (warp & 3) * 32 + lane;
+    const int elh = erow / a.TW, elw = erow - elh * a.TW;
+    const int sexp = s_rowsexp[erow];
+    const bool valid = sexp != INT_MIN && !dead;
+    const bool bad = sexp == INT_MAX;
+    long long S = 0;
+    double inv = 0.0;
+    if (valid && !bad) {
+      long long s4[4];
+#pragma unroll
+      for (int p = 0; p < 4; ++p) s4[p] = (long long)s_rowsum[0][erow][p] + (long long)s_rowsum[1][erow][p];
+      S = (s4[3] << 24) + (s4[2] << 16) + (s4[1] << 8) + s4[0];
+      inv = __hiloint2double((1023 - sexp) << 20, 0);
+    }
+    const double Sd = (double)S;
+    const int64_t plane_hw = (int64_t)a.Ho * a.Wo;
+    const int64_t obase = (int64_t)img * a.d.Cout * plane_hw + (int64_t)(ho0 + elh) * a.Wo + (wo0 + elw);
+    const int cb = warp >> 2;
+#pragma unroll 1
+    for (int c8 = 0; c8 < 4; ++c8) {
+      const int col = cb * 32 + c8 * 8;
+      uint32_t v[4][8];
+      const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col;
+#pragma unroll
+      for (int p = 0; p < 4; ++p) tmem_load_8(taddr + (uint32_t)(p * WB_NT), v[p]);
+      tmem_load_wait();
+      if (!valid) continue;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const int j = col + jj;
+        if (j0 + j >= a.d.Cout) break;
+        float out;
+        if (bad) {
+          out = __uint_as_float(0x7FC00000u);
+        } else {
+          const long long M1 = ((long long)(int)v[3][jj] << 24) + ((long long)(int)v[2][jj] << 16) +
+                               ((long long)(int)v[1][jj] << 8) + (long long)(int)v[0][jj];
+          const double m1 = (double)M1, m0 = Sd - m1;  // exact: |.| < 2^45
+          const double y = __dadd_rn(__dmul_rn(s_alpha[j], m1), __dmul_rn(s_beta[j], m0));
+          out = (float)__dmul_rn(y, inv);
+        }
+        a.y[obase + (int64_t)(j0 + j) * plane_hw] = out;
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 4 * WB_NT);
+}
+
+uint32_t magic_for(uint32_t d) { return d > 1 ? (uint32_t)((0x100000000ull + d - 1) / d) : 0u; }
+
+}  // namespace
+
+cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, const uint32_t* wmask,
+                             int32_t ldw, const float* walpha, const float* wbeta, float* y, cudaStream_t stream) {
+  WbinArgs a;
+  a.d = d; a.Ho = Ho; a.Wo = Wo;
+  a.khw = d.kh * d.kw;
+  a.n = d.C * a.khw;
+  a.words = (a.n + 31) / 32;
+  a.x = x; a.wmask = wmask; a.ldw = ldw; a.walpha = walpha; a.wbeta = wbeta; a.y = y;
+  // Tile: rows of at most 16 output positions, as many rows as fit the 128 lanes, both evened out over the image.
+  const int tw_tiles = (Wo + 15) / 16;
+  a.TW = (Wo + tw_tiles - 1) / tw_tiles;
+  int TH = std::min(Ho, kLanes / a.TW);
+  const size_t fixed = 4 * (size_t)WB_PLANE + WB_BSTAGE + 128;
+  const size_t limit2 = 110 * 1024, limit1 = 227 * 1024 - 8 * 1024;  // two CTAs per SM / one
+  a.max_ch = std::min(d.C, (WB_KS + a.khw - 1) / a.khw + 1);
+  size_t smem = 0;
+  for (;;) {
+    const int th_tiles = (Ho + TH - 1) / TH;
+    a.TH = (Ho + th_tiles - 1) / th_tiles;
+    a.in_h = (a.TH - 1) * d.stride_h + d.kh;
+    a.in_w = (a.TW - 1) * d.stride_w + d.kw;
+    a.pitch = a.in_w | 1;
+    a.ch_words = a.in_h * a.pitch;
+    smem = fixed + sizeof(float) * (size_t)a.max_ch * a.ch_words + sizeof(uint32_t) * (size_t)a.in_h * a.in_w;
+    const bool offsets_fit = (size_t)a.max_ch * a.ch_words < kNoElement;
+    if ((smem <= limit2 && offsets_fit) || TH == 1) break;
+    TH = a.TH - 1;
+  }
+  if (smem > limit1 || (size_t)a.max_ch * a.ch_words >= kNoElement) return cudaErrorInvalidValue;
+  a.tiles_h = (Ho + a.TH - 1) / a.TH;
+  a.tiles_w = (Wo + a.TW - 1) / a.TW;
+  a.magic_npix = magic_for((uint32_t)(a.in_h * a.in_w));
+  a.magic_in_w = magic_for((uint32_t)a.in_w);
+  a.magic_khw = magic_for((uint32_t)a.khw);
+  a.magic_kw = magic_for((uint32_t)d.kw);
+  const int64_t gx = (int64_t)d.N * a.tiles_h * a.tiles_w;
+  const int64_t gy = (d.Cout + WB_NT - 1) / WB_NT;
+  if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(wbin_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  wbin_conv_kernel<<<dim3((unsigned)gx, (unsigned)gy), WB_THREADS, smem, stream>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t read_wbin_wait_timeouts(unsigned int* count) {
+  return cudaMemcpyFromSymbol(count, g_wbin_wait_timeouts, sizeof(unsigned int));
+}
+
+}  // namespace dab
