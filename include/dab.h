@@ -177,7 +177,9 @@ dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, con
  *   y[img][co][ho][wo] = alpha_co * (sum of the patch values under e_co) + beta_co * (sum of the others),
  * with nothing done to the activations.  Patch definition, element order (c, kh, kw), zero padding and output
  * layout as in dab_binary_conv; the filters come from dab_binarize on the [Cout x C*kh*kw] weight matrix
- * (their K is not needed).  No workspace.
+ * (their K is not needed).
+ *   d_workspace, workspace_bytes   scratch of at least dab_wbin_conv_workspace(desc) bytes (one word per input
+ *                                  pixel: the largest magnitude over its channels), 256-byte aligned
  *
  * Arithmetic: each patch is taken as 32-bit fixed point relative to its own largest magnitude and the sums
  * under e are formed exactly in integers on the tensor cores, so the result differs from exact arithmetic by
@@ -186,8 +188,10 @@ dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, con
  * in all its outputs.  C*H*W must be below 2^31.
  * DAB_ERR_UNSUPPORTED if no tile of the layer fits shared memory (kernels wider than about 200 columns).
  */
+size_t dab_wbin_conv_workspace(const dab_conv_desc* desc);
 dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
-                         const float* d_walpha, const float* d_wbeta, float* d_y, void* stream);
+                         const float* d_walpha, const float* d_wbeta, float* d_y, void* d_workspace,
+                         size_t workspace_bytes, void* stream);
 
 /*
  * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up

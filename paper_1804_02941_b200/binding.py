@@ -24,7 +24,7 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
-           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv")
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace")
 
 
 class DabError(RuntimeError):
@@ -71,7 +71,9 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_static_capacity.argtypes = []
         L.dab_binary_conv_static.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
-        L.dab_wbin_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
+        L.dab_wbin_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
+        L.dab_wbin_conv_workspace.restype = C.c_size_t
+        L.dab_wbin_conv_workspace.argtypes = [vp]
         L.dab_set_contraction.argtypes = [i32]
         L.dab_get_contraction.argtypes = []
         L.dab_contraction_wait_failures.argtypes = [vp]
@@ -320,9 +322,13 @@ def dab_binary_conv_static(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(
     return y
 
 
+def dab_wbin_conv_workspace(desc: ConvDesc) -> int:
+    return int(lib().dab_wbin_conv_workspace(C.byref(desc)))
+
+
 def dab_wbin_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
-                  y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
-    """Weights-only binarized convolution: fp32 NCHW input against the two-level filters `w` (no workspace)."""
+                  y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Weights-only binarized convolution: fp32 NCHW input against the two-level filters `w`."""
     _dev(x, torch.float32, "x")
     if not x.is_contiguous():
         raise ValueError("x must be contiguous NCHW")
@@ -331,8 +337,11 @@ def dab_wbin_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pa
     Ho, Wo = dab_conv_output_size(desc)
     if y is None:
         y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=x.device)
+    need = dab_wbin_conv_workspace(desc)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
     st = lib().dab_wbin_conv(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.alpha), _ptr(w.beta), _ptr(y),
-                             _stream(stream))
+                             _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "dab_wbin_conv")
     return y
 

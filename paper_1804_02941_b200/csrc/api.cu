@@ -386,8 +386,15 @@ dab_status dab_contraction_wait_failures(uint32_t* h_count) {
   return from_cuda(e);
 }
 
+size_t dab_wbin_conv_workspace(const dab_conv_desc* desc) {
+  ConvGeom g;
+  if (!conv_geom(desc, &g)) return 0;
+  return round_up((size_t)desc->N * desc->H * desc->W * sizeof(uint32_t), kAlign);
+}
+
 dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
-                         const float* d_walpha, const float* d_wbeta, float* d_y, void* stream) {
+                         const float* d_walpha, const float* d_wbeta, float* d_y, void* d_workspace,
+                         size_t workspace_bytes, void* stream) {
   if (!desc) return DAB_ERR_INVALID_ARG;
   if (desc->C > 0 && desc->kh > 0 && desc->kw > 0 && (int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N)
     return DAB_ERR_UNSUPPORTED;
@@ -396,8 +403,12 @@ dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint
   if (!d_x || !d_wmask || !d_walpha || !d_wbeta || !d_y) return DAB_ERR_INVALID_ARG;
   if (ldw < dab_words_per_row(g.n) || (ldw & 3) || !aligned16(d_wmask)) return DAB_ERR_INVALID_ARG;
   if (desc->Cout > 65535 * 64 || (int64_t)desc->C * desc->H * desc->W > 0x7FFFFFFF) return DAB_ERR_UNSUPPORTED;
+  if ((int64_t)desc->N * desc->H * desc->W > (int64_t)0x7FFFFFFF * 256) return DAB_ERR_UNSUPPORTED;
+  if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign) ||
+      workspace_bytes < dab_wbin_conv_workspace(desc))
+    return DAB_ERR_WORKSPACE;
   cudaError_t e = launch_wbin_conv(*desc, g.Ho, g.Wo, d_x, d_wmask, ldw, d_walpha, d_wbeta, d_y,
-                                   static_cast<cudaStream_t>(stream));
+                                   static_cast<uint32_t*>(d_workspace), static_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return DAB_ERR_UNSUPPORTED;  // no tile of this layer fits shared memory
   return from_cuda(e);
 }

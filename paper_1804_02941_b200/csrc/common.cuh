@@ -96,9 +96,11 @@ cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64
 cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
                                 float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
                                 cudaStream_t stream);
-// Weights-only binarized convolution on the tensor cores; see wbin.cu.  cudaErrorInvalidValue: no tile fits.
+// Weights-only binarized convolution on the tensor cores; see wbin.cu.  pixmax: N*H*W words of scratch.
+// cudaErrorInvalidValue: no tile fits.
 cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, const uint32_t* wmask,
-                             int32_t ldw, const float* walpha, const float* wbeta, float* y, cudaStream_t stream);
+                             int32_t ldw, const float* walpha, const float* wbeta, float* y, uint32_t* pixmax,
+                             cudaStream_t stream);
 cudaError_t read_wbin_wait_timeouts(unsigned int* count);
 cudaError_t launch_popc_probe(uint32_t* sink, int32_t blocks, int32_t iters, cudaStream_t stream);
 

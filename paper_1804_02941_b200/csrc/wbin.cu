@@ -35,7 +35,6 @@ constexpr int WB_NT = 64;                        // filters per CTA
 constexpr uint32_t WB_SBO = WB_KC * 128;         // bytes between groups of 8 rows
 constexpr uint32_t WB_PLANE = kLanes * WB_KS;    // bytes of one byte plane of the activation stage
 constexpr uint32_t WB_BSTAGE = WB_NT * WB_KS;    // bytes of the filter stage
-constexpr uint16_t kNoElement = 0xFFFFu;
 
 struct WbinArgs {
   dab_conv_desc d;
@@ -44,6 +43,7 @@ struct WbinArgs {
   int32_t in_h, in_w, pitch, ch_words, max_ch;
   uint32_t magic_npix, magic_in_w, magic_khw, magic_kw;  // ceil(2^32 / d): floor(i / d) = umulhi(i, magic); 0 if d == 1
   const float* x;
+  const uint32_t* pixmax;  // N x H x W: largest magnitude over the channels, as a bit pattern
   const uint32_t* wmask;
   int32_t ldw;
   const float* walpha;
@@ -65,6 +65,38 @@ __device__ __forceinline__ void byte_planes(uint32_t q0, uint32_t q1, uint32_t q
   out[3] = __byte_perm(b, d, 0x7632);
 }
 
+// Sixteen consecutive elements (K chunk kc of the stage) of one row: gathered through the offset table, scaled
+// by 2^sexp in two exact steps, rounded to 32-bit integers, split into byte planes and stored as one 16-byte K
+// chunk per plane; the byte sums of the planes accumulate in psum.  kChecked: elements from `limit` on are 0.
+template <bool kChecked>
+__device__ __forceinline__ void gather_chunk(const float* src, const uint16_t* off, int kc, int limit, float fac,
+                                             float fac2, unsigned char* dst0, int (&psum)[4]) {
+  uint32_t pl[4][4];
+#pragma unroll
+  for (int g4 = 0; g4 < 4; ++g4) {
+    uint32_t q[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int kk = kc * 16 + g4 * 4 + e;
+      float v = src[off[kk]];
+      if (kChecked && kk >= limit) v = 0.0f;
+      q[e] = (uint32_t)__float2int_rn(__fmul_rn(__fmul_rn(v, fac), fac2));
+    }
+    uint32_t w4[4];
+    byte_planes(q[0], q[1], q[2], q[3], w4);
+#pragma unroll
+    for (int p = 0; p < 4; ++p) pl[p][g4] = w4[p];
+    psum[0] = (int)__dp4a(w4[0], 0x01010101u, (unsigned)psum[0]);
+    psum[1] = (int)__dp4a(w4[1], 0x01010101u, (unsigned)psum[1]);
+    psum[2] = (int)__dp4a(w4[2], 0x01010101u, (unsigned)psum[2]);
+    psum[3] = __dp4a((int)w4[3], 0x01010101, psum[3]);
+  }
+  unsigned char* dst = dst0 + (uint32_t)kc * 128;
+#pragma unroll
+  for (int p = 0; p < 4; ++p)
+    *reinterpret_cast<uint4*>(dst + p * WB_PLANE) = make_uint4(pl[p][0], pl[p][1], pl[p][2], pl[p][3]);
+}
+
 __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs a) {
   extern __shared__ __align__(128) unsigned char dyn_mem[];
   __shared__ __align__(8) uint64_t s_bar;
@@ -72,14 +104,16 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
   __shared__ int s_rowsexp[kLanes];      // scale exponent of a row; INT_MIN: row not in the image; INT_MAX: non-finite
   __shared__ int s_rowsum[2][kLanes][4]; // byte-plane sums of q over the row, one set per gathering thread
   __shared__ double s_alpha[WB_NT], s_beta[WB_NT];
-  __shared__ uint16_t s_off[WB_KS];
+  __shared__ uint16_t s_off[2][WB_KS];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t mem0 = (smem_u32(dyn_mem) + 127u) & ~127u;
   unsigned char* const stage_a = dyn_mem + (mem0 - smem_u32(dyn_mem));
   unsigned char* const stage_b = stage_a + 4 * WB_PLANE;
-  float* const tile = reinterpret_cast<float*>(stage_b + WB_BSTAGE);
-  uint32_t* const pixmax = reinterpret_cast<uint32_t*>(tile + (size_t)a.max_ch * a.ch_words);
+  // two input tiles: the next group of channels arrives while the current one is gathered
+  const int tile_words = a.max_ch * a.ch_words;
+  float* const tiles = reinterpret_cast<float*>(stage_b + WB_BSTAGE);
+  uint32_t* const pixmax = reinterpret_cast<uint32_t*>(tiles + 2 * (size_t)tile_words);
   const uint32_t bar = smem_u32(&s_bar);
 
   // tile of this CTA
@@ -101,18 +135,14 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
     s_alpha[j] = in ? (double)a.walpha[j0 + j] : 0.0;
     s_beta[j] = in ? (double)a.wbeta[j0 + j] : 0.0;
   }
-  for (int p = tid; p < npix; p += WB_THREADS) pixmax[p] = 0u;
-  __syncthreads();
-
-  // Largest magnitude over the channels of every staged pixel (as bit patterns: NaN > Inf > finite).
-  for (int idx = tid; idx < a.d.C * npix; idx += WB_THREADS) {
-    const int c = fast_div(idx, a.magic_npix), pix = idx - c * npix;
+  // per-pixel maxima of the staged region (0 outside the image)
+  for (int pix = tid; pix < npix; pix += WB_THREADS) {
     const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
     const int h = h0 + r, w = w0 + s;
-    if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W) {
-      const uint32_t m = __float_as_uint(__ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w)) & 0x7FFFFFFFu;
-      if (m) atomicMax(&pixmax[pix], m);
-    }
+    uint32_t m = 0u;
+    if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
+      m = __ldg(a.pixmax + ((int64_t)img * a.d.H + h) * a.d.W + w);
+    pixmax[pix] = m;
   }
   __syncthreads();
 
@@ -149,29 +179,44 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
   bool dead = false;
   uint32_t parity = 0;
   const int stages = (a.words + WB_JS - 1) / WB_JS;
-  for (int st = 0; st < stages; ++st) {
-    const int k0 = st * WB_KS;
-    const int k1 = min(a.n, k0 + WB_KS);
+  // Asynchronous copy of the channels that stage `st` draws from into tile buffer st & 1, and the offsets of its
+  // elements inside that tile.
+  auto stage_in = [&](int st) {
+    const int k0 = st * WB_KS, k1 = min(a.n, k0 + WB_KS);
     const int c_lo = fast_div(k0, a.magic_khw), c_hi = fast_div(k1 - 1, a.magic_khw) + 1;
-    // (1) stage the channels this group of elements comes from; offsets of the elements inside the staged tile
+    float* const tile = tiles + (st & 1) * tile_words;
     for (int idx = tid; idx < (c_hi - c_lo) * npix; idx += WB_THREADS) {
       const int c = fast_div(idx, a.magic_npix), pix = idx - c * npix;
       const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
       const int h = h0 + r, w = w0 + s;
-      float v = 0.0f;
-      if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
-        v = __ldg(ximg + ((int64_t)(c_lo + c) * a.d.H + h) * a.d.W + w);
-      tile[c * a.ch_words + r * a.pitch + s] = v;
+      const bool in = (unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W;
+      const float* src = in ? ximg + ((int64_t)(c_lo + c) * a.d.H + h) * a.d.W + w : ximg;
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(tile + c * a.ch_words + r * a.pitch + s)),
+                   "l"(src), "r"(in ? 4 : 0)
+                   : "memory");  // source size 0: the word is filled with zeros
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
     if (tid < WB_KS) {
       const int k = k0 + tid;
-      uint16_t o = kNoElement;
+      int o = 0;  // beyond the patch length: any staged word (the gather replaces it by 0)
       if (k < a.n) {
         const int c = fast_div(k, a.magic_khw), rs = k - c * a.khw;
         const int r = fast_div(rs, a.magic_kw), s = rs - r * a.d.kw;
-        o = (uint16_t)((c - c_lo) * a.ch_words + r * a.pitch + s);
+        o = (c - c_lo) * a.ch_words + r * a.pitch + s;
       }
-      s_off[tid] = o;
+      s_off[st & 1][tid] = (uint16_t)o;
+    }
+  };
+
+  stage_in(0);
+  for (int st = 0; st < stages; ++st) {
+    const int k0 = st * WB_KS;
+    // (1) start the copy for the next stage; wait for this stage's own
+    if (st + 1 < stages) {
+      stage_in(st + 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
     // (2) the tensor cores have finished reading the previous contents of the operand stages
@@ -181,34 +226,18 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
     }
     // (3) gather, convert, split into byte planes: thread = (row, every other 16-element chunk)
     if (gather) {
-      const float* const src = tile + origin;
+      const float* const src = tiles + (st & 1) * tile_words + origin;
+      const uint16_t* const off = s_off[st & 1];
+      unsigned char* const dst0 = stage_a + (uint32_t)(row >> 3) * WB_SBO + (row & 7) * 16;
+      if (k0 + WB_KS <= a.n) {
 #pragma unroll
-      for (int t = 0; t < WB_KC / 2; ++t) {
-        const int kc = half + 2 * t;
-        if (k0 + kc * 16 >= a.n) break;
-        uint32_t pl[4][4];
-#pragma unroll
-        for (int g4 = 0; g4 < 4; ++g4) {
-          uint32_t q[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const uint16_t o = s_off[kc * 16 + g4 * 4 + e];
-            const float v = (o != kNoElement) ? src[o] : 0.0f;
-            q[e] = (uint32_t)__float2int_rn(__fmul_rn(__fmul_rn(v, fac), fac2));
-          }
-          uint32_t w4[4];
-          byte_planes(q[0], q[1], q[2], q[3], w4);
-#pragma unroll
-          for (int p = 0; p < 4; ++p) pl[p][g4] = w4[p];
-          psum[0] = (int)__dp4a(w4[0], 0x01010101u, (unsigned)psum[0]);
-          psum[1] = (int)__dp4a(w4[1], 0x01010101u, (unsigned)psum[1]);
-          psum[2] = (int)__dp4a(w4[2], 0x01010101u, (unsigned)psum[2]);
-          psum[3] = __dp4a((int)w4[3], 0x01010101, psum[3]);
+        for (int t = 0; t < WB_KC / 2; ++t) gather_chunk<false>(src, off, half + 2 * t, 0, fac, fac2, dst0, psum);
+      } else {  // last stage of a row length that is not a multiple of 128: elements beyond it count as 0
+        for (int t = 0; t < WB_KC / 2; ++t) {
+          const int kc = half + 2 * t;
+          if (k0 + kc * 16 >= a.n) break;
+          gather_chunk<true>(src, off, kc, a.n - k0, fac, fac2, dst0, psum);
         }
-        unsigned char* dst = stage_a + (uint32_t)(row >> 3) * WB_SBO + (uint32_t)kc * 128 + (row & 7) * 16;
-#pragma unroll
-        for (int p = 0; p < 4; ++p)
-          *reinterpret_cast<uint4*>(dst + p * WB_PLANE) = make_uint4(pl[p][0], pl[p][1], pl[p][2], pl[p][3]);
       }
     }
     // (4) the masks of the 64 filters: four words of a row -> eight K chunks of 0/1 bytes
@@ -294,13 +323,35 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
   if (warp == 0) tmem_dealloc(tmem, 4 * WB_NT);
 }
 
+// Largest magnitude over the channels of every pixel, as a bit pattern (NaN > Inf > finite): what the
+// convolution kernel derives the scale of a patch from.  One thread per pixel, coalesced along the image.
+__global__ void __launch_bounds__(256) wbin_pixmax_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
+                                                          int C, int64_t HW, int64_t total) {
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= total) return;
+  const int64_t img = idx / HW, p = idx - img * HW;
+  const float* src = x + img * C * HW + p;
+  uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
+  int c = 0;
+  for (; c + 4 <= C; c += 4) {
+    m0 = max(m0, __float_as_uint(__ldg(src + (int64_t)c * HW)) & 0x7FFFFFFFu);
+    m1 = max(m1, __float_as_uint(__ldg(src + (int64_t)(c + 1) * HW)) & 0x7FFFFFFFu);
+    m2 = max(m2, __float_as_uint(__ldg(src + (int64_t)(c + 2) * HW)) & 0x7FFFFFFFu);
+    m3 = max(m3, __float_as_uint(__ldg(src + (int64_t)(c + 3) * HW)) & 0x7FFFFFFFu);
+  }
+  for (; c < C; ++c) m0 = max(m0, __float_as_uint(__ldg(src + (int64_t)c * HW)) & 0x7FFFFFFFu);
+  out[idx] = max(max(m0, m1), max(m2, m3));
+}
+
 uint32_t magic_for(uint32_t d) { return d > 1 ? (uint32_t)((0x100000000ull + d - 1) / d) : 0u; }
 
 }  // namespace
 
 cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, const uint32_t* wmask,
-                             int32_t ldw, const float* walpha, const float* wbeta, float* y, cudaStream_t stream) {
+                             int32_t ldw, const float* walpha, const float* wbeta, float* y, uint32_t* pixmax,
+                             cudaStream_t stream) {
   WbinArgs a;
+  a.pixmax = pixmax;
   a.d = d; a.Ho = Ho; a.Wo = Wo;
   a.khw = d.kh * d.kw;
   a.n = d.C * a.khw;
@@ -321,12 +372,12 @@ cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, con
     a.in_w = (a.TW - 1) * d.stride_w + d.kw;
     a.pitch = a.in_w | 1;
     a.ch_words = a.in_h * a.pitch;
-    smem = fixed + sizeof(float) * (size_t)a.max_ch * a.ch_words + sizeof(uint32_t) * (size_t)a.in_h * a.in_w;
-    const bool offsets_fit = (size_t)a.max_ch * a.ch_words < kNoElement;
+    smem = fixed + 2 * sizeof(float) * (size_t)a.max_ch * a.ch_words + sizeof(uint32_t) * (size_t)a.in_h * a.in_w;
+    const bool offsets_fit = (size_t)a.max_ch * a.ch_words <= 65535;
     if ((smem <= limit2 && offsets_fit) || TH == 1) break;
     TH = a.TH - 1;
   }
-  if (smem > limit1 || (size_t)a.max_ch * a.ch_words >= kNoElement) return cudaErrorInvalidValue;
+  if (smem > limit1 || (size_t)a.max_ch * a.ch_words > 65535) return cudaErrorInvalidValue;
   a.tiles_h = (Ho + a.TH - 1) / a.TH;
   a.tiles_w = (Wo + a.TW - 1) / a.TW;
   a.magic_npix = magic_for((uint32_t)(a.in_h * a.in_w));
@@ -336,7 +387,11 @@ cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, con
   const int64_t gx = (int64_t)d.N * a.tiles_h * a.tiles_w;
   const int64_t gy = (d.Cout + WB_NT - 1) / WB_NT;
   if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(wbin_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const int64_t HW = (int64_t)d.H * d.W, pixels = (int64_t)d.N * HW;
+  wbin_pixmax_kernel<<<(unsigned)((pixels + 255) / 256), 256, 0, stream>>>(x, pixmax, d.C, HW, pixels);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(wbin_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   wbin_conv_kernel<<<dim3((unsigned)gx, (unsigned)gy), WB_THREADS, smem, stream>>>(a);
   return cudaGetLastError();

@@ -118,10 +118,16 @@ def test_rejects_bad_arguments(dab):
     L = dab.lib()
     desc = dab.make_desc((1, 4, 8, 8), 4, 3, 3, (1, 1), (1, 1))
     import ctypes as C
-    assert L.dab_wbin_conv(C.byref(desc), None, None, 4, None, None, None, None) == 1
+    assert L.dab_wbin_conv(C.byref(desc), None, None, 4, None, None, None, None, 0, None) == 1
     x = torch.zeros((1, 4, 8, 8), device="cuda")
     m = torch.zeros((4, 4), dtype=torch.int32, device="cuda")
     a = torch.zeros(4, device="cuda")
     y = torch.zeros((1, 4, 8, 8), device="cuda")
-    assert L.dab_wbin_conv(C.byref(desc), x.data_ptr(), m.data_ptr(), 1, a.data_ptr(), a.data_ptr(), y.data_ptr(), None) == 1
-    assert L.dab_wbin_conv(C.byref(desc), x.data_ptr(), m.data_ptr(), 6, a.data_ptr(), a.data_ptr(), y.data_ptr(), None) == 1
+    ws = torch.zeros(dab.dab_wbin_conv_workspace(desc), dtype=torch.uint8, device="cuda")
+    args = (x.data_ptr(), m.data_ptr())
+    tail = (a.data_ptr(), a.data_ptr(), y.data_ptr())
+    assert L.dab_wbin_conv(C.byref(desc), *args, 1, *tail, ws.data_ptr(), ws.numel(), None) == 1       # ld too short
+    assert L.dab_wbin_conv(C.byref(desc), *args, 6, *tail, ws.data_ptr(), ws.numel(), None) == 1       # ld not a multiple of 4
+    assert L.dab_wbin_conv(C.byref(desc), *args, 4, *tail, ws.data_ptr(), ws.numel() - 1, None) == 3   # scratch too small
+    assert L.dab_wbin_conv(C.byref(desc), *args, 4, *tail, None, ws.numel(), None) == 3
+    assert L.dab_wbin_conv(C.byref(desc), *args, 4, *tail, ws.data_ptr(), ws.numel(), None) == 0
