@@ -55,6 +55,7 @@ def parse_args():
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-wbin", action="store_true", help="skip the weights-only binarized pass over the same layers")
     return ap.parse_args()
 
 
@@ -396,6 +397,32 @@ def run_dab(args):
         e2e = {"value": aggregate_throughput(ops_per_step, args.e2e_steps, e2e_s, world) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * e2e_s / args.e2e_steps}
 
+    # The paper's weights-only binarized networks on the same layers: fp32 activations against the coded filters
+    # (dab_wbin_conv, four int8 tensor-core products per multiply-accumulate).  Reported beside the headline, not in it.
+    wbin = None
+    if not args.no_wbin:
+        wws = torch.empty(max(dab.dab_wbin_conv_workspace(desc) for (_, _, _, _, desc, _, _) in work), dtype=torch.uint8, device=dev)
+
+        def wbin_step():
+            for (L, x, w, wc, desc, pm, y) in work:
+                dab.dab_wbin_conv(x, wc, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad), y=y, workspace=wws, stream=stream)
+        for _ in range(3):
+            wbin_step()
+        stream.synchronize()
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0.record(stream)
+        for _ in range(args.steps):
+            wbin_step()
+        w1.record(stream)
+        stream.synchronize()
+        wms = w0.elapsed_time(w1) / args.steps
+        int8_peak, int8_src = load_int8_peak()
+        macs = ops_per_step / 2
+        wbin = {"kernel": "wbin_conv_kernel (+ wbin_pixmax_kernel)", "ms_per_step": wms, "tmacs": macs / wms / 1e9,
+                "bound": "tensor", "achieved": 8 * macs / wms / 1e9, "unit": "int8 TOPS (4 byte planes x 2 ops per MAC)",
+                "peak": int8_peak, "frac": 8 * macs / wms / 1e9 / int8_peak, "peak_source": int8_src,
+                "gpu_launches": 2 * len(work) * args.steps}
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         b = args.cpu_sample_batch
@@ -413,7 +440,7 @@ def run_dab(args):
                "gpu_launches": 3 * launches_per_kind,
                "kernel_ms_per_step": {k: v / args.steps for k, v in k_ms.items()},
                "binarize_gbs": binarize_gbs, "roofline": roofline, "roofline_contraction": roofline_contract,
-               "cpu_baseline": cpu_baseline, "contraction_wait_failures": dab.dab_contraction_wait_failures()}
+               "wbin": wbin, "cpu_baseline": cpu_baseline, "contraction_wait_failures": dab.dab_contraction_wait_failures()}
         print(json.dumps(out))
     if world > 1:
         import torch.distributed as dist

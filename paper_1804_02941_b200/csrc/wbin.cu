@@ -68,7 +68,8 @@ __device__ __forceinline__ void byte_planes(uint32_t q0, uint32_t q1, uint32_t q
 // Sixteen consecutive elements (K chunk kc of the stage) of one row: gathered through the offset table, scaled
 // by 2^sexp in two exact steps, rounded to 32-bit integers, split into byte planes and stored as one 16-byte K
 // chunk per plane; the byte sums of the planes accumulate in psum.  kChecked: elements from `limit` on are 0.
-template <bool kChecked>
+// kTwoStep: the scale is beyond one fp32 factor (patches whose largest magnitude is below 2^-70).
+template <bool kChecked, bool kTwoStep>
 __device__ __forceinline__ void gather_chunk(const float* src, const uint16_t* off, int kc, int limit, float fac,
                                              float fac2, unsigned char* dst0, int (&psum)[4]) {
   uint32_t pl[4][4];
@@ -80,7 +81,9 @@ __device__ __forceinline__ void gather_chunk(const float* src, const uint16_t* o
       const int kk = kc * 16 + g4 * 4 + e;
       float v = src[off[kk]];
       if (kChecked && kk >= limit) v = 0.0f;
-      q[e] = (uint32_t)__float2int_rn(__fmul_rn(__fmul_rn(v, fac), fac2));
+      v = __fmul_rn(v, fac);
+      if (kTwoStep) v = __fmul_rn(v, fac2);
+      q[e] = (uint32_t)__float2int_rn(v);
     }
     uint32_t w4[4];
     byte_planes(q[0], q[1], q[2], q[3], w4);
@@ -229,14 +232,14 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
       const float* const src = tiles + (st & 1) * tile_words + origin;
       const uint16_t* const off = s_off[st & 1];
       unsigned char* const dst0 = stage_a + (uint32_t)(row >> 3) * WB_SBO + (row & 7) * 16;
-      if (k0 + WB_KS <= a.n) {
+      if (k0 + WB_KS <= a.n && sexp2 == 0) {
 #pragma unroll
-        for (int t = 0; t < WB_KC / 2; ++t) gather_chunk<false>(src, off, half + 2 * t, 0, fac, fac2, dst0, psum);
-      } else {  // last stage of a row length that is not a multiple of 128: elements beyond it count as 0
+        for (int t = 0; t < WB_KC / 2; ++t) gather_chunk<false, false>(src, off, half + 2 * t, 0, fac, fac2, dst0, psum);
+      } else {  // a row length that is not a multiple of 128 (elements beyond it count as 0) or a two-step scale
         for (int t = 0; t < WB_KC / 2; ++t) {
           const int kc = half + 2 * t;
           if (k0 + kc * 16 >= a.n) break;
-          gather_chunk<true>(src, off, kc, a.n - k0, fac, fac2, dst0, psum);
+          gather_chunk<true, true>(src, off, kc, a.n - k0, fac, fac2, dst0, psum);
         }
       }
     }

@@ -50,7 +50,17 @@ def emit(**kw):
     print(json.dumps(kw), flush=True)
 
 
+STAGES = None   # set of stage names to run (--stages), None: all
+LAYERS = None   # set of layer names to run (--layers), None: all
+
+
+def want_stage(name):
+    return STAGES is None or name in STAGES
+
+
 def conv_layer(cfg, L, stream, hbm, tops_peak, dense=False):
+    if LAYERS is not None and L.name not in LAYERS:
+        return
     dev = torch.device("cuda")
     x = torch.from_numpy(L.inputs(stream=stream, dense=dense)).to(dev)
     w = torch.from_numpy(L.weights(stream=stream)).to(dev)
@@ -61,20 +71,39 @@ def conv_layer(cfg, L, stream, hbm, tops_peak, dense=False):
     pg, pd = torch.empty(P, device=dev), torch.empty(P, device=dev)
     pm = torch.empty((P, ld), dtype=torch.int32, device=dev)
     y = torch.empty((L.N, L.Cout, L.Ho, L.Wo), device=dev)
-    t_w = timed(lambda: dab.dab_binarize_into(w, wd.K, wd.alpha, wd.beta, wd.mask, wd.flags))
-    t_s = timed(lambda: dab.dab_sign_patches(desc, x, pK, pg, pd, pm, None))   # FBin-style input coding, for comparison
-    t_p = timed(lambda: dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, None))
-    t_c = timed(lambda: dab.dab_binary_conv_contract(desc, pm, pK, pg, pd, wd, y, None))
     wd_words = dab.dab_words_per_row(L.n)
     bytes_p = 4 * x.numel() + P * (4 * wd_words + 12)
     bytes_w = L.Cout * (4 * L.n + 4 * wd_words + 12)
     common = dict(config=cfg, layer=L.name, n=L.n, patches=P, filters=L.Cout, inputs="dense" if dense else "relu60")
-    emit(stage="binarize_filters", ms=t_w, gbs=bytes_w / t_w / 1e6, hbm_frac=bytes_w / t_w / 1e6 / hbm, **common)
-    emit(stage="binarize_patches", ms=t_p, gbs=bytes_p / t_p / 1e6, hbm_frac=bytes_p / t_p / 1e6 / hbm, **common)
-    emit(stage="sign_patches", ms=t_s, gbs=bytes_p / t_s / 1e6, hbm_frac=bytes_p / t_s / 1e6 / hbm, **common)
-    emit(stage="contract", ms=t_c, tops_equiv=L.binary_ops / t_c / 1e9, alu_frac=L.binary_ops / t_c / 1e9 / tops_peak,
-         **common)
-    emit(stage="conv_total", ms=t_p + t_c, tops_equiv=L.binary_ops / (t_p + t_c) / 1e9, **common)
+    if want_stage("binarize_filters"):
+        t_w = timed(lambda: dab.dab_binarize_into(w, wd.K, wd.alpha, wd.beta, wd.mask, wd.flags))
+        emit(stage="binarize_filters", ms=t_w, gbs=bytes_w / t_w / 1e6, hbm_frac=bytes_w / t_w / 1e6 / hbm, **common)
+    if want_stage("sign_patches"):   # FBin-style input coding, for comparison
+        t_s = timed(lambda: dab.dab_sign_patches(desc, x, pK, pg, pd, pm, None))
+        emit(stage="sign_patches", ms=t_s, gbs=bytes_p / t_s / 1e6, hbm_frac=bytes_p / t_s / 1e6 / hbm, **common)
+    t_p = t_c = None
+    if want_stage("binarize_patches") or want_stage("contract"):
+        t_p = timed(lambda: dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, None))
+        emit(stage="binarize_patches", ms=t_p, gbs=bytes_p / t_p / 1e6, hbm_frac=bytes_p / t_p / 1e6 / hbm, **common)
+    if want_stage("contract"):
+        t_c = timed(lambda: dab.dab_binary_conv_contract(desc, pm, pK, pg, pd, wd, y, None))
+        emit(stage="contract", ms=t_c, tops_equiv=L.binary_ops / t_c / 1e9, alu_frac=L.binary_ops / t_c / 1e9 / tops_peak,
+             **common)
+        emit(stage="conv_total", ms=t_p + t_c, tops_equiv=L.binary_ops / (t_p + t_c) / 1e9, **common)
+    if want_stage("wbin_conv"):
+        # weights-only binarized layer: fp32 activations x two-level filters, four int8 tensor-core products per MAC
+        ws = torch.empty(dab.dab_wbin_conv_workspace(desc), dtype=torch.uint8, device=dev)
+        t_b = timed(lambda: dab.dab_wbin_conv(x, wd, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad), y=y, workspace=ws))
+        macs = L.binary_ops / 2
+        emit(stage="wbin_conv", ms=t_b, tmacs=macs / t_b / 1e9, int8_tops=8 * macs / t_b / 1e9,
+             int8_frac=8 * macs / t_b / 1e9 / int8_peak(), **common)
+
+
+def int8_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return 2.0 * float(json.load(open(p))["bf16_tflops_sustained"])
+    return 2800.0
 
 
 def gemm_point(m, k, hbm, tops_peak):
@@ -115,7 +144,12 @@ def main():
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--batch5", type=int, default=256)
     ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"])
+    ap.add_argument("--stages", default="", help="comma-separated stage names of the convolution layers to run (default all)")
+    ap.add_argument("--layers", default="", help="comma-separated layer names to run (default all)")
     args = ap.parse_args()
+    global STAGES, LAYERS
+    STAGES = set(args.stages.split(",")) if args.stages else None
+    LAYERS = set(args.layers.split(",")) if args.layers else None
     dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
     want = set(args.configs.split(","))
     hbm, mhz, src = peaks()

@@ -131,3 +131,37 @@ def test_rejects_bad_arguments(dab):
     assert L.dab_wbin_conv(C.byref(desc), *args, 4, *tail, ws.data_ptr(), ws.numel() - 1, None) == 3   # scratch too small
     assert L.dab_wbin_conv(C.byref(desc), *args, 4, *tail, None, ws.numel(), None) == 3
     assert L.dab_wbin_conv(C.byref(desc), *args, 4, *tail, ws.data_ptr(), ws.numel(), None) == 0
+
+
+@pytest.mark.parametrize("name", ["l1_0", "l2_0", "l2_1", "l3_1", "l4_0", "l4_1"])
+def test_config5_layers_at_batch_256_on_sampled_images(dab, name):
+    # the launch the sweep times (whole layer, batch 256); the checker recomputes three whole images of it
+    from dab_synth import configs
+    L = next(l for l in configs.config5(256) if l.name == name)
+    x, w = L.inputs(stream=11), L.weights(stream=11)
+    wb = oracle.binarize(w)
+    got = dab.dab_wbin_conv(to_dev(x), dab.dab_binarize(to_dev(w)), L.kh, L.kw, (L.stride,) * 2, (L.pad,) * 2)
+    torch.cuda.synchronize()
+    assert dab.dab_contraction_wait_failures() == 0
+    assert bool(torch.isfinite(got).all())
+    for img in (0, 131, 255):
+        ref, mag = oracle.conv_wbin(x[img:img + 1], wb.e, wb.alpha, wb.beta, L.kh, L.kw, (L.stride,) * 2, (L.pad,) * 2)
+        err = np.abs(got[img:img + 1].cpu().numpy().astype(np.float64) - ref)
+        assert np.all(err <= 1e-5 * mag + 1e-300)
+        assert np.all(err <= 2.0 ** -31 * L.n * float(np.abs(x[img]).max()) * float(np.abs(np.r_[wb.alpha, wb.beta]).max())
+                      + 2.0 ** -23 * np.abs(ref))
+
+
+def test_config4_and_config2_shapes(dab):
+    # 5x5 and 6x6 / 7x7 kernels, 1x1 "fully connected" layers, batch 1 and batch 128
+    from dab_synth import configs
+    for L in list(configs.config2()) + [configs.config4(128)[i] for i in (0, 4, 5)]:
+        x, w = L.inputs(stream=12), L.weights(stream=12)
+        sel = slice(0, min(L.N, 2))
+        wb = oracle.binarize(w)
+        got = dab.dab_wbin_conv(to_dev(x), dab.dab_binarize(to_dev(w)), L.kh, L.kw, (L.stride,) * 2, (L.pad,) * 2)
+        torch.cuda.synchronize()
+        ref, mag = oracle.conv_wbin(x[sel], wb.e, wb.alpha, wb.beta, L.kh, L.kw, (L.stride,) * 2, (L.pad,) * 2)
+        err = np.abs(got[sel].cpu().numpy().astype(np.float64) - ref)
+        assert np.all(err <= 1e-5 * mag + 1e-300), L.name
+    assert dab.dab_contraction_wait_failures() == 0
