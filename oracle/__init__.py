@@ -193,6 +193,34 @@ def conv_wbin(x, w_e, w_alpha, w_beta, kh, kw, stride=(1, 1), pad=(0, 0)):
     return y, mag
 
 
+def train_forward(W: np.ndarray):
+    """Algorithm 2, steps 4-13: returns (Wc, Binarized of Wc, Wt dense)."""
+    W = np.ascontiguousarray(W, np.float32)
+    rows, n = W.shape
+    Wc, Wt = np.zeros_like(W), np.zeros_like(W)
+    e = np.zeros((rows, n), np.uint8)
+    K, flags = np.zeros(rows, np.int32), np.zeros(rows, np.uint32)
+    alpha, beta = np.zeros(rows, np.float32), np.zeros(rows, np.float32)
+    lib().oracle_train_forward(_p(W), C.c_int64(rows), C.c_int32(n), _p(Wc), _p(e), _p(K), _p(alpha), _p(beta),
+                               _p(flags), _p(Wt))
+    return Wc, e, K, alpha, beta, flags, Wt
+
+
+def theorem4(Wc: np.ndarray, e: np.ndarray, K: np.ndarray, grad_Wt: np.ndarray | None = None):
+    """Theorem 4: returns (G fp64, grad_W fp32 or None)."""
+    Wc = np.ascontiguousarray(Wc, np.float32)
+    e = np.ascontiguousarray(e, np.uint8)
+    K = np.ascontiguousarray(K, np.int32)
+    rows, n = Wc.shape
+    G = np.zeros((rows, n), np.float64)
+    gw = None
+    if grad_Wt is not None:
+        grad_Wt = np.ascontiguousarray(grad_Wt, np.float32)
+        gw = np.zeros((rows, n), np.float32)
+    lib().oracle_theorem4(_p(Wc), _p(e), _p(K), C.c_int64(rows), C.c_int32(n), _p(G), _p(grad_Wt), _p(gw))
+    return G, gw
+
+
 def im2col(x, kh, kw, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     """Patch rows (N*Ho*Wo) x (C*kh*kw), element order (c, kh, kw), zero padding as 0.0 values."""
     x = np.ascontiguousarray(x, np.float32)

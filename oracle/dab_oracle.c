@@ -324,3 +324,59 @@ void oracle_conv_wbin(const oracle_conv_desc* d, const float* x, const uint8_t* 
     free(p);
   }
 }
+
+/* Algorithm 2, steps 4-13 for the filters of one layer: MeanCenter (the mean of the filter's n weights is
+ * subtracted), Clamp to [-1, 1], then Algorithm 1 and the dense two-level filter of Corollary 1. */
+void oracle_train_forward(const float* W, int64_t rows, int32_t n, float* Wc, uint8_t* e, int32_t* K, float* alpha,
+                          float* beta, uint32_t* flags, float* Wt) {
+  int64_t r;
+  for (r = 0; r < rows; ++r) {
+    const float* w = W + r * (int64_t)n;
+    float* c = Wc + r * (int64_t)n;
+    double sum = 0.0, mean;
+    int32_t i;
+    for (i = 0; i < n; ++i) sum = sum + (double)w[i];
+    mean = sum / (double)n;
+    for (i = 0; i < n; ++i) {
+      float v = (float)((double)w[i] - mean);
+      if (v > 1.0f) v = 1.0f;
+      if (v < -1.0f) v = -1.0f;
+      c[i] = v;
+    }
+    oracle_binarize_row(c, n, e + r * (int64_t)n, K + r, alpha + r, beta + r, flags + r, 0, 0, 0);
+    if (Wt)
+      for (i = 0; i < n; ++i) Wt[r * (int64_t)n + i] = e[r * (int64_t)n + i] ? alpha[r] : beta[r];
+  }
+}
+
+/* Theorem 4, element by element, for rows W (the mean-centred, clamped weights that were coded) with masks e:
+ *   T_k = W o e (the selected weights, zeros elsewhere), sgn(T_k) read as the membership indicator e,
+ *   sgn(W - T_k) as 1 - e, STE(V)_i = V_i where |W_i| <= 1 and 0 elsewhere;
+ *   G1_i = e_i / K + (||T_k||_1 / K) * STE(T_k)_i
+ *   G2_i = (1 - e_i) / (n - K) + (||W - T_k||_1 / (n - K)) * STE(W - T_k)_i
+ *   G = G1 + G2 (fp64).  Rows with K = 0 (constant rows) get G = 0.
+ * grad_W (nullable) = grad_Wt o G rounded to fp32: the gradient handed to the weight update. */
+void oracle_theorem4(const float* W, const uint8_t* e, const int32_t* K, int64_t rows, int32_t n, double* G,
+                     const float* grad_Wt, float* grad_W) {
+  int64_t r;
+  for (r = 0; r < rows; ++r) {
+    const float* w = W + r * (int64_t)n;
+    const uint8_t* m = e + r * (int64_t)n;
+    double l1_sel = 0.0, l1_rest = 0.0;
+    int32_t i, k = K[r];
+    for (i = 0; i < n; ++i) {
+      if (m[i]) l1_sel = l1_sel + fabs((double)w[i]);
+      else l1_rest = l1_rest + fabs((double)w[i]);
+    }
+    for (i = 0; i < n; ++i) {
+      double g = 0.0;
+      if (k > 0 && k < n) {
+        double ste = (fabs((double)w[i]) <= 1.0) ? (double)w[i] : 0.0;
+        if (m[i]) g = 1.0 / (double)k + (l1_sel / (double)k) * ste;
+        else g = 1.0 / (double)(n - k) + (l1_rest / (double)(n - k)) * ste;
+      }
+      if (G) G[r * (int64_t)n + i] = g;
+      if (grad_W) grad_W[r * (int64_t)n + i] = (float)((double)grad_Wt[r * (int64_t)n + i] * g);
+    }
+  }
+}

@@ -9,7 +9,8 @@
  *
  * Every function below is pinned by CPU tests against something other than
  * itself (exhaustive search over all masks, direct sums of squared error, closed
- * forms, a library im2col, a textbook XNOR-popcount); none is "parity unpinned".
+ * forms, a library im2col, a textbook XNOR-popcount).  One exception, marked "PARITY UNPINNED" at its
+ * declaration: the straight-through terms of oracle_theorem4.
  */
 #ifndef DAB_ORACLE_H
 #define DAB_ORACLE_H
@@ -105,6 +106,26 @@ void oracle_conv_sign(const oracle_conv_desc* d, const float* x, const uint8_t* 
  */
 void oracle_conv_wbin(const oracle_conv_desc* d, const float* x, const uint8_t* w_e, const float* w_alpha,
                       const float* w_beta, float* y, double* abs_terms);
+
+/*
+ * Algorithm 2, steps 4-13 (binarizing the weight filters of one layer during training):
+ *   Wc = Clamp(MeanCenter(W), -1, 1): the mean of each filter's n weights (fp64 sum in element order, divided by
+ *   n) is subtracted in fp64, the difference rounded to fp32 and clamped;  (e, K, alpha, beta) = Algorithm 1 on Wc;
+ *   Wt (nullable) = alpha e + beta (1 - e), the dense filter of Corollary 1.  All arrays rows x n, dense.
+ */
+void oracle_train_forward(const float* W, int64_t rows, int32_t n, float* Wc, uint8_t* e, int32_t* K, float* alpha,
+                          float* beta, uint32_t* flags, float* Wt);
+
+/*
+ * Theorem 4 (backward pass), element by element; W is the mean-centred, clamped weight matrix that was coded.
+ *   G (nullable, fp64, rows x n) = G1 + G2 as printed, with sgn(T_k) read as the membership indicator e;
+ *   grad_W (nullable) = grad_Wt o G rounded to fp32.  See the comment in the source for every term.
+ * PARITY UNPINNED for the two STE terms: the paper prints them without a definition they could be checked
+ * against (they are not the derivative of anything the paper defines); the other two terms are pinned as the
+ * derivatives of alpha and beta with e held fixed.
+ */
+void oracle_theorem4(const float* W, const uint8_t* e, const int32_t* K, int64_t rows, int32_t n, double* G,
+                     const float* grad_Wt, float* grad_W);
 
 /* Patch extraction alone (explicit loops), rows = N*Ho*Wo, row length C*kh*kw. */
 void oracle_im2col(const oracle_conv_desc* d, const float* x, float* patches);
