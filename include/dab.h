@@ -194,6 +194,29 @@ dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint
                          size_t workspace_bytes, void* stream);
 
 /*
+ * dab_binarize_train — Algorithm 2, steps 4-13: how the filters of a layer are binarized at every training
+ * step.  For each row (filter) of d_W:
+ *   Wc = Clamp(MeanCenter(W), -1, 1)   the mean of the row's n weights (fp64) is subtracted, the result rounded
+ *                                      to fp32 and clamped; Wc is what Algorithm 2 keeps as W_real and what is coded
+ *   (e, K, alpha, beta) = Algorithm 1 on Wc, exactly as dab_binarize
+ *   Wt = alpha e + beta (1 - e)        the dense filter of Corollary 1 (d_Wt may be NULL)
+ * d_W, d_Wc, d_Wt: rows x n fp32 with row strides ld_* (floats); d_Wc may not alias d_W unless ld_Wc == ld_W
+ * (then the update is in place).  The other arguments are those of dab_binarize.
+ *
+ * dab_binarize_backward — Theorem 4: grad_W = grad_Wt o G, the gradient handed to the weight update, with
+ *   G_i = e_i / K + (||T_k||_1 / K) STE(T_k)_i + (1 - e_i) / (n - K) + (||W - T_k||_1 / (n - K)) STE(W - T_k)_i,
+ * T_k = Wc o e, STE(V)_i = V_i where |Wc_i| <= 1 and 0 elsewhere, sgn(T_k) of the printed formula read as the
+ * membership indicator e.  d_Wc, d_mask, d_K are the outputs of dab_binarize_train; rows with K = 0 (constant
+ * rows) get a zero gradient.  fp64 internally, one rounding to fp32.
+ */
+dab_status dab_binarize_train(const float* d_W, int64_t rows, int32_t n, int64_t ld_W, float* d_Wc, int64_t ld_Wc,
+                              float* d_Wt, int64_t ld_Wt, int32_t* d_K, float* d_alpha, float* d_beta,
+                              uint32_t* d_mask, int32_t ld_mask, uint32_t* d_row_flags, void* stream);
+dab_status dab_binarize_backward(const float* d_Wc, int64_t rows, int32_t n, int64_t ld_Wc, const uint32_t* d_mask,
+                                 int32_t ld_mask, const int32_t* d_K, const float* d_grad_Wt, int64_t ld_grad_Wt,
+                                 float* d_grad_W, int64_t ld_grad_W, void* stream);
+
+/*
  * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up
  * to 16 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
  * chunks overlap on three streams, and the call returns after everything has drained.  Use pinned host memory:

@@ -24,7 +24,7 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
-           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace")
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward")
 
 
 class DabError(RuntimeError):
@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
         L.dab_wbin_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
         L.dab_wbin_conv_workspace.restype = C.c_size_t
         L.dab_wbin_conv_workspace.argtypes = [vp]
+        L.dab_binarize_train.argtypes = [vp, i64, i32, i64, vp, i64, vp, i64, vp, vp, vp, vp, i32, vp, vp]
+        L.dab_binarize_backward.argtypes = [vp, i64, i32, i64, vp, i32, vp, vp, i64, vp, i64, vp]
         L.dab_set_contraction.argtypes = [i32]
         L.dab_get_contraction.argtypes = []
         L.dab_contraction_wait_failures.argtypes = [vp]
@@ -344,6 +346,39 @@ def dab_wbin_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pa
                              _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "dab_wbin_conv")
     return y
+
+
+def dab_binarize_train(W: torch.Tensor, want_dense: bool = True, stream=None):
+    """Algorithm 2 steps 4-13 on the rows of W: returns (Wc, Coded of Wc, Wt or None)."""
+    _dev(W, torch.float32, "W")
+    if W.dim() != 2 or W.stride(1) != 1:
+        raise ValueError("W must be a 2-D tensor with contiguous rows")
+    rows, n = W.shape
+    ld = dab_default_ld(n)
+    dev = W.device
+    Wc = torch.empty((rows, n), dtype=torch.float32, device=dev)
+    Wt = torch.empty((rows, n), dtype=torch.float32, device=dev) if want_dense else None
+    out = Coded(torch.empty((rows, ld), dtype=torch.int32, device=dev), torch.empty(rows, dtype=torch.int32, device=dev),
+                torch.empty(rows, dtype=torch.float32, device=dev), torch.empty(rows, dtype=torch.float32, device=dev),
+                torch.empty(rows, dtype=torch.int32, device=dev), n)
+    st = lib().dab_binarize_train(_ptr(W), rows, n, W.stride(0) if rows > 1 else n, _ptr(Wc), n, _ptr(Wt), n, _ptr(out.K),
+                                  _ptr(out.alpha), _ptr(out.beta), _ptr(out.mask), ld, _ptr(out.flags), _stream(stream))
+    _check(st, "dab_binarize_train")
+    return Wc, out, Wt
+
+
+def dab_binarize_backward(Wc: torch.Tensor, coded: Coded, grad_Wt: torch.Tensor, stream=None) -> torch.Tensor:
+    """Theorem 4: the gradient with respect to the real-valued weights from the gradient with respect to W~."""
+    _dev(Wc, torch.float32, "Wc")
+    _dev(grad_Wt, torch.float32, "grad_Wt")
+    rows, n = Wc.shape
+    if not (Wc.is_contiguous() and grad_Wt.is_contiguous() and grad_Wt.shape == Wc.shape):
+        raise ValueError("Wc and grad_Wt must be contiguous and of one shape")
+    gW = torch.empty_like(Wc)
+    st = lib().dab_binarize_backward(_ptr(Wc), rows, n, n, _ptr(coded.mask), coded.ld, _ptr(coded.K), _ptr(grad_Wt), n,
+                                     _ptr(gW), n, _stream(stream))
+    _check(st, "dab_binarize_backward")
+    return gW
 
 
 def dab_popc_probe(blocks: int, iters: int, sink: torch.Tensor | None = None, stream=None) -> torch.Tensor:

@@ -413,6 +413,32 @@ dab_status dab_wbin_conv(const dab_conv_desc* desc, const float* d_x, const uint
   return from_cuda(e);
 }
 
+dab_status dab_binarize_train(const float* d_W, int64_t rows, int32_t n, int64_t ld_W, float* d_Wc, int64_t ld_Wc,
+                              float* d_Wt, int64_t ld_Wt, int32_t* d_K, float* d_alpha, float* d_beta,
+                              uint32_t* d_mask, int32_t ld_mask, uint32_t* d_row_flags, void* stream) {
+  if (rows < 0 || n < 1) return DAB_ERR_INVALID_ARG;
+  if (n > DAB_MAX_N) return DAB_ERR_UNSUPPORTED;
+  if (ld_W < n || ld_Wc < n || (d_Wt && ld_Wt < n) || ld_mask < dab_words_per_row(n) || (ld_mask & 3))
+    return DAB_ERR_INVALID_ARG;
+  if (rows == 0) return DAB_OK;
+  if (!d_W || !d_Wc || !d_K || !d_alpha || !d_beta || !d_mask || !aligned16(d_mask)) return DAB_ERR_INVALID_ARG;
+  return from_cuda(launch_train_forward(d_W, rows, n, ld_W, d_Wc, ld_Wc, d_Wt, ld_Wt, d_K, d_alpha, d_beta, d_mask,
+                                        ld_mask, d_row_flags, static_cast<cudaStream_t>(stream)));
+}
+
+dab_status dab_binarize_backward(const float* d_Wc, int64_t rows, int32_t n, int64_t ld_Wc, const uint32_t* d_mask,
+                                 int32_t ld_mask, const int32_t* d_K, const float* d_grad_Wt, int64_t ld_grad_Wt,
+                                 float* d_grad_W, int64_t ld_grad_W, void* stream) {
+  if (rows < 0 || n < 1) return DAB_ERR_INVALID_ARG;
+  if (n > DAB_MAX_N) return DAB_ERR_UNSUPPORTED;
+  if (ld_Wc < n || ld_grad_Wt < n || ld_grad_W < n || ld_mask < dab_words_per_row(n) || (ld_mask & 3))
+    return DAB_ERR_INVALID_ARG;
+  if (rows == 0) return DAB_OK;
+  if (!d_Wc || !d_mask || !d_K || !d_grad_Wt || !d_grad_W) return DAB_ERR_INVALID_ARG;
+  return from_cuda(launch_train_backward(d_Wc, ld_Wc, d_mask, ld_mask, d_K, rows, n, d_grad_Wt, ld_grad_Wt, d_grad_W,
+                                         ld_grad_W, static_cast<cudaStream_t>(stream)));
+}
+
 dab_status dab_popc_probe(uint32_t* d_sink, int32_t blocks, int32_t iters, void* stream) {
   if (!d_sink || blocks < 1 || iters < 0) return DAB_ERR_INVALID_ARG;
   return from_cuda(launch_popc_probe(d_sink, blocks, iters, static_cast<cudaStream_t>(stream)));

@@ -102,6 +102,13 @@ cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, con
                              int32_t ldw, const float* walpha, const float* wbeta, float* y, uint32_t* pixmax,
                              cudaStream_t stream);
 cudaError_t read_wbin_wait_timeouts(unsigned int* count);
+// Training-side weight binarization and its gradient factor; see train.cu.  Wt may be null.
+cudaError_t launch_train_forward(const float* W, int64_t rows, int32_t n, int64_t ld_W, float* Wc, int64_t ld_Wc,
+                                 float* Wt, int64_t ld_Wt, int32_t* K, float* alpha, float* beta, uint32_t* mask,
+                                 int32_t ld_mask, uint32_t* flags, cudaStream_t stream);
+cudaError_t launch_train_backward(const float* Wc, int64_t ld_Wc, const uint32_t* mask, int32_t ld_mask,
+                                  const int32_t* K, int64_t rows, int32_t n, const float* gWt, int64_t ld_g, float* gW,
+                                  int64_t ld_gw, cudaStream_t stream);
 cudaError_t launch_popc_probe(uint32_t* sink, int32_t blocks, int32_t iters, cudaStream_t stream);
 
 }  // namespace dab
