@@ -24,7 +24,7 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
-           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward")
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward", "dab_set_patch_coder", "dab_get_patch_coder")
 
 
 class DabError(RuntimeError):
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
         L.dab_binarize_train.argtypes = [vp, i64, i32, i64, vp, i64, vp, i64, vp, vp, vp, vp, i32, vp, vp]
         L.dab_binarize_backward.argtypes = [vp, i64, i32, i64, vp, i32, vp, vp, i64, vp, i64, vp]
         L.dab_set_contraction.argtypes = [i32]
+        L.dab_set_patch_coder.argtypes = [i32]
+        L.dab_get_patch_coder.argtypes = []
         L.dab_get_contraction.argtypes = []
         L.dab_contraction_wait_failures.argtypes = [vp]
         _lib = L
@@ -394,6 +396,18 @@ CONTRACT_AUTO, CONTRACT_TENSOR, CONTRACT_POPC = 0, 1, 2
 def dab_set_contraction(path: int) -> None:
     """Process-wide choice of the contraction kernel: CONTRACT_AUTO (default), CONTRACT_TENSOR or CONTRACT_POPC."""
     _check(lib().dab_set_contraction(int(path)), "dab_set_contraction")
+
+
+PATCHES_SORT, PATCHES_HIST = 0, 1
+
+
+def dab_set_patch_coder(coder: int) -> None:
+    """PATCHES_SORT (default: full sort per patch) or PATCHES_HIST (histogram-pruned search where it applies)."""
+    _check(lib().dab_set_patch_coder(int(coder)), "dab_set_patch_coder")
+
+
+def dab_get_patch_coder() -> int:
+    return int(lib().dab_get_patch_coder())
 
 
 def dab_get_contraction() -> int:

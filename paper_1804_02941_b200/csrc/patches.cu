@@ -198,6 +198,375 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Histogram-pruned patch coder.  One warp per patch, three passes over the patch in the staged tile:
+//   1. every non-zero value is quantised (q = floor(v * qscale), a fixed scale per tile) and counted into one of
+//      B = 32*BPL buckets (bucket = high bits of q): per bucket the count and the sum of the low bits of q, by
+//      shared-memory atomics;
+//   2. a scan over the buckets gives, at every bucket edge, the split size s exactly and the prefix sum P to
+//      within the quantisation error, hence the objective there to within a known eps; inside a bucket the
+//      objective is bounded by its values at the corners of the parallelogram that the bucket's value range
+//      allows (the objective is jointly convex in (s, P)).  Buckets whose bound cannot reach the best edge value
+//      are discarded; the hull of the others (usually two or three buckets) is gathered, with exact fp64 sums of
+//      everything below and above it, sorted and searched by the exact evaluator of rowcode.cuh;
+//   3. the mask is a threshold compare, as in the other coders.
+// Discarding is conservative (every rounding is covered by eps), so the result is the same split the full
+// search finds.  Patches whose hull exceeds 256 values, and tiles holding a NaN or an infinity, are left to the
+// group kernel through the dense-tile mark.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kHistCap = 256;  // keys the exact search takes at most
+
+struct HistTile {          // per tile, in shared memory
+  uint32_t kmin, kmax;     // smallest and largest key among the non-zero staged values
+  int retry;               // some patch of the tile could not be coded here
+};
+
+__device__ __forceinline__ float objective_f32(float s, float P, float T, float n) {
+  // P^2/s + (T-P)^2/(n-s) with the limits 0 at s = 0 (P = 0 there) and s = n
+  const float Q = T - P;
+  const float a = s > 0.0f ? __fdividef(P * P, s) : 0.0f;
+  const float b = n - s > 0.0f ? __fdividef(Q * Q, n - s) : 0.0f;
+  return a + b;
+}
+
+template <int E>
+__device__ __noinline__ RowResult hist_sort_select(const uint32_t* scratch, int m, int z, int n, int lane,
+                                                   const double* rcp, const SplitBase base) {
+  uint32_t r[E];
+#pragma unroll
+  for (int j = 0; j < E; ++j) {
+    const int idx = j * 32 + lane;
+    r[j] = idx < m ? order_key(__uint_as_float(scratch[idx])) : kPadKey;   // the gather stored raw bits
+  }
+  group_sort<1, E>(r, lane, nullptr, 0);
+  return group_select<1, E, true, true>(r, m, z, n, lane, nullptr, 0, rcp, base);
+}
+
+#ifndef DAB_HIST_MINBLOCKS
+#define DAB_HIST_MINBLOCKS 3  // CTAs per SM the histogram coder is compiled for (register budget)
+#endif
+
+// KHW: kh*kw when it is 9 (the sweeps over a patch are then fully unrolled over the kernel window), 0 otherwise.
+template <int BPL, int KHW>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binarize_patches_hist_kernel(const PatchArgs a) {
+  constexpr int THREADS = kWarpsPerCta * 32;
+  constexpr int B = 32 * BPL;
+  constexpr int LOG2B = BPL == 1 ? 5 : BPL == 2 ? 6 : BPL == 4 ? 7 : 8;
+  constexpr int KMAX = KHW ? KHW : 1;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* rcp = reinterpret_cast<double*>(smem_raw);
+  int2* hist_all = reinterpret_cast<int2*>(rcp + rcp_table_slots(a.n));          // [warp][B] (count, sum of offsets)
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(hist_all + kWarpsPerCta * B);
+  float* tile = reinterpret_cast<float*>(scratch_all + kWarpsPerCta * kHistCap);
+  const int ch_words = (a.in_h * a.pitch) | 1;  // odd: the 32 channels a warp reads at once fall into 32 banks
+  uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
+  uint16_t* win = off + ((a.n + 1) & ~1);       // offsets of the kernel window inside one channel
+  __shared__ HistTile ht;
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int2* hist = hist_all + warp * B;
+  uint32_t* scratch = scratch_all + warp * kHistCap;
+  const int khw = a.d.kh * a.d.kw;
+  fill_reciprocals(rcp, a.n, threadIdx.x, THREADS);
+  fill_offsets(a, off, ch_words, threadIdx.x, THREADS);
+  for (int rs = threadIdx.x; rs < khw; rs += THREADS) win[rs] = (uint16_t)((rs / a.d.kw) * a.pitch + rs % a.d.kw);
+  __syncthreads();
+  int wofs[KMAX];
+#pragma unroll
+  for (int rs = 0; rs < KMAX; ++rs) wofs[rs] = KHW ? win[rs] : 0;
+  // bits of q: 24 (fp32 holds them), fewer if the sum of n in-bucket offsets (qbits - log2 B bits each) could leave 32 bits
+  int qbits = 24;
+  while (((int64_t)a.n << (qbits - LOG2B)) >= 0x7FFFFFFFll) --qbits;
+  const int rounds = (a.n + 31) >> 5;
+  const float nf = (float)a.n;
+  const unsigned lt = (1u << lane) - 1u;
+
+  const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+    const TileCoord t = tile_coord(a, tile_id);
+    __syncthreads();  // the previous tile is no longer read
+    if (threadIdx.x == 0) { ht.kmin = kPadKey; ht.kmax = 0u; ht.retry = 0; }
+    __syncthreads();
+    {  // stage the values (-0.0 folded onto +0.0) and find the range of the non-zero ones
+      const float* ximg = a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W;
+      const int per_ch = a.in_h * a.in_w, total = a.d.C * per_ch;
+      uint32_t kmin = kPadKey, kmax = 0u;
+      for (int idx = threadIdx.x; idx < total; idx += THREADS) {
+        int c = a.magic_per_ch ? (int)__umulhi((unsigned)idx, a.magic_per_ch) : idx;
+        int rem = idx - c * per_ch;
+        int r = a.magic_in_w ? (int)__umulhi((unsigned)rem, a.magic_in_w) : rem;
+        int s = rem - r * a.in_w;
+        int h = t.h0 + r, w = t.w0 + s;
+        float v = 0.0f;
+        if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
+          v = __fadd_rn(__ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w), 0.0f);
+        tile[c * ch_words + r * a.pitch + s] = v;
+        if (v != 0.0f) {  // NaN compares unequal: counted, and seen as non-finite below
+          const uint32_t key = order_key(v);
+          kmin = min(kmin, key);
+          kmax = max(kmax, key);
+        }
+      }
+      kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+      kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+      if (lane == 0 && kmin <= kmax) {
+        atomicMin(&ht.kmin, kmin);
+        atomicMax(&ht.kmax, kmax);
+      }
+    }
+    __syncthreads();
+    const int64_t first_patch = ((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0;
+    const uint32_t tkmin = ht.kmin, tkmax = ht.kmax;
+    const bool any_nonzero = tkmin <= tkmax;
+    if (any_nonzero && key_range_nonfinite(tkmin, tkmax)) {
+      if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+      continue;
+    }
+    // Quantisation of the tile: q = floor(v * qscale); bucket = (q >> shift) + boff; B0 = first bucket of positives.
+    const float lo = any_nonzero ? key_value(tkmin) : 0.0f, hi = any_nonzero ? key_value(tkmax) : 0.0f;
+    float qscale;
+    int boff, B0;
+    const int shift = qbits - LOG2B;
+    if (lo >= 0.0f) {         // no negative value: q in [0, 2^qbits)
+      qscale = __fdividef((float)(1 << qbits) * 0.99999f, fmaxf(hi, 1e-37f));
+      boff = 0; B0 = 0;
+    } else if (hi <= 0.0f) {  // no positive value: q in [-2^qbits, 0)
+      qscale = __fdividef((float)(1 << qbits) * 0.99999f, -lo);
+      boff = B; B0 = B;
+    } else {                  // both signs: q in [-2^(qbits-1), 2^(qbits-1))
+      qscale = __fdividef((float)(1 << (qbits - 1)) * 0.99999f, fmaxf(-lo, hi));
+      boff = B / 2; B0 = B / 2;
+    }
+    const float u = __fdividef(1.0f, qscale);              // value of one unit of q
+    const int qmask = (1 << shift) - 1;
+    const float bw = (float)(1 << shift);                  // bucket width in units of q
+    const float A = fmaxf(fabsf(lo), fabsf(hi)), R = hi - lo;
+
+    for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
+      const int lh = p / t.tw, lw = p % t.tw;
+      const float* origin = tile + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+      const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
+      uint32_t* mrow = a.pmask + pi * (int64_t)a.ldp;
+
+      // ---- pass 1: histogram (the order of the elements does not matter: lane = channel, loop over the window) ----
+#pragma unroll
+      for (int j = 0; j < BPL; ++j) hist[lane * BPL + j] = make_int2(0, 0);
+      __syncwarp();
+      for (int c0 = 0; c0 < a.d.C; c0 += 32) {
+        const bool cin = c0 + lane < a.d.C;
+        const float* src = origin + (cin ? c0 + lane : 0) * ch_words;
+        auto tally = [&](float v) {
+          const int q = __float2int_rd(v * qscale);
+          const int b = min(max((q >> shift) + boff, 0), B - 1);
+          if (cin && v != 0.0f) {
+            atomicAdd(&hist[b].x, 1);
+            atomicAdd(&hist[b].y, q & qmask);
+          }
+        };
+        if (KHW) {
+#pragma unroll
+          for (int rs = 0; rs < KMAX; ++rs) tally(src[wofs[rs]]);
+        } else {
+          for (int rs = 0; rs < khw; ++rs) tally(src[win[rs]]);
+        }
+      }
+      __syncwarp();
+      // ---- scan over the buckets: lane owns buckets lane*BPL .. lane*BPL+BPL-1 ----
+      int c[BPL];
+      double Q[BPL];   // sum of q over the bucket: count * first q of the bucket + sum of the offsets (exact)
+      int csum = 0;
+      double qsum = 0.0;
+#pragma unroll
+      for (int j = 0; j < BPL; ++j) {
+        const int2 hq = hist[lane * BPL + j];
+        c[j] = hq.x;
+        Q[j] = (double)hq.x * (double)((lane * BPL + j - boff) * (1 << shift)) + (double)(unsigned)hq.y;
+        csum += hq.x; qsum += Q[j];
+      }
+      int cincl = csum;
+      double qincl = qsum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int co = __shfl_up_sync(0xFFFFFFFFu, cincl, o);
+        const double qo = __shfl_up_sync(0xFFFFFFFFu, qincl, o);
+        if (lane >= o) { cincl += co; qincl += qo; }
+      }
+      const int m = __shfl_sync(0xFFFFFFFFu, cincl, 31);
+      const double QT = __shfl_sync(0xFFFFFFFFu, qincl, 31);
+      const int z = a.n - m;
+      RowResult res;
+      bool retry = false;
+      if (m == 0) {
+        res = trivial_row(false, 0.0f);  // nothing but zeros
+      } else {
+        // nominal prefix sums in units of u: every value lies in [(q - 1) u, (q + 2) u], centre (q + 0.5) u
+        const float Tn = ((float)QT + 0.5f * (float)m) * u;
+        const float eps_fixed = 3.0f * (R + A) * (float)m * u;          // effect of the quantisation on any objective value
+        int cbefore = cincl - csum;
+        double qbefore = qincl - qsum;
+        float best_edge = -1.0f;
+        float bound[BPL];
+        int negc_local = 0;
+#pragma unroll
+        for (int j = 0; j < BPL; ++j) {
+          const int b = lane * BPL + j;
+          const float s0 = (float)(cbefore + (b >= B0 ? z : 0));
+          const float P0 = ((float)qbefore + 0.5f * (float)cbefore) * u;
+          const int cafter = cbefore + c[j];
+          const double qafter = qbefore + Q[j];
+          const float s1 = s0 + (float)c[j];
+          const float P1 = ((float)qafter + 0.5f * (float)cafter) * u;
+          float d0 = -1.0f, d1 = -1.0f, dk = -1.0f;
+          if (s0 > 0.0f && s0 < nf) d0 = objective_f32(s0, P0, Tn, nf);
+          if (s1 > 0.0f && s1 < nf) d1 = objective_f32(s1, P1, Tn, nf);
+          best_edge = fmaxf(best_edge, fmaxf(d0, d1));
+          if (c[j] >= 2) {
+            // value range of the bucket, and the two inner corners of the region (s, P) can visit inside it
+            const float qlo = (float)(b - boff) * bw;
+            const float va = (qlo - 1.0f) * u, vb = (qlo + bw + 2.0f) * u;
+            const float cf = (float)c[j], sig = P1 - P0;
+            float jl = __fdividef(cf * vb - sig, vb - va);
+            jl = fminf(fmaxf(jl, 0.0f), cf);
+            const float ju = cf - jl;
+            dk = fmaxf(objective_f32(s0 + jl, P0 + jl * va, Tn, nf), objective_f32(s0 + ju, P0 + ju * vb, Tn, nf));
+            // the corners move with the uncertainty of the bucket's sum: 1.5 c u in P, that over (vb - va) in s
+            dk += (A * A + 2.0f * R * A) * __fdividef(1.5f * cf * u, vb - va) + 2.0f * R * 1.5f * cf * u;
+          }
+          bound[j] = c[j] > 0 ? fmaxf(fmaxf(d0, d1), dk) : -2.0f;
+          if (b < B0) negc_local += c[j];
+          cbefore = cafter; qbefore = qafter;
+        }
+        const int negc = __reduce_add_sync(0xFFFFFFFFu, negc_local);
+        // the two splits around the run of zeros (their sums are those of the negatives)
+        const double qneg = __shfl_sync(0xFFFFFFFFu, qincl, max(B0 / BPL - 1, 0));   // inclusive sum up to bucket B0-1
+        const float Pneg = B0 > 0 ? ((float)qneg + 0.5f * (float)negc) * u : 0.0f;
+        float dz0 = -1.0f, dz1 = -1.0f;
+        if (z > 0) {
+          if (negc > 0) dz0 = objective_f32((float)negc, Pneg, Tn, nf);
+          if (negc + z < a.n) dz1 = objective_f32((float)(negc + z), Pneg, Tn, nf);
+        }
+        best_edge = fmaxf(best_edge, fmaxf(dz0, dz1));
+        best_edge = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fmaxf(best_edge, 0.0f))));
+        // a bucket (or the zero run) survives if its bound, raised by every rounding, reaches the best edge lowered by them
+        const float slack = 2.0f * eps_fixed + 2e-4f * best_edge;
+        const float need = best_edge - slack;
+        int seg_lo = 1 << 20, seg_hi = -1;
+#pragma unroll
+        for (int j = 0; j < BPL; ++j) {
+          const int b = lane * BPL + j;
+          if (c[j] > 0 && bound[j] + slack >= need) {
+            const int seg = b + (b >= B0 ? 1 : 0);
+            seg_lo = min(seg_lo, seg);
+            seg_hi = max(seg_hi, seg);
+          }
+        }
+        if (z > 0 && fmaxf(dz0, dz1) + slack >= need) { seg_lo = min(seg_lo, B0); seg_hi = max(seg_hi, B0); }
+        seg_lo = __reduce_min_sync(0xFFFFFFFFu, seg_lo);
+        seg_hi = __reduce_max_sync(0xFFFFFFFFu, seg_hi);
+        // hull in bucket and q terms
+        const int b_lo = seg_lo > B0 ? seg_lo - 1 : seg_lo;          // first bucket of the hull (seg_lo == B0: bucket B0)
+        const int b_hi = seg_hi >= B0 ? seg_hi - 1 : seg_hi;         // last bucket of the hull (seg_hi == B0: bucket B0-1)
+        const int z_in = (z > 0 && seg_lo <= B0 && B0 <= seg_hi) ? z : 0;
+        int msub_local = 0, sbelow_local = 0;
+#pragma unroll
+        for (int j = 0; j < BPL; ++j) {
+          const int b = lane * BPL + j;
+          if (b >= b_lo && b <= b_hi) msub_local += c[j];
+          if (b < b_lo) sbelow_local += c[j];
+        }
+        const int m_sub = __reduce_add_sync(0xFFFFFFFFu, msub_local);
+        int s_below = __reduce_add_sync(0xFFFFFFFFu, sbelow_local);
+        if (seg_lo > B0) s_below += z;                               // the zeros lie below the hull
+        // (a constant row has all its values in one bucket: with more than kHistCap values it is left to the group kernel)
+        if (seg_hi < 0 || m_sub < 1 || m_sub > kHistCap || (z == 0 && m_sub == a.n)) {
+          retry = true;
+        } else {
+          const int qA = (b_lo - boff) * (1 << shift);               // q range of the hull's buckets
+          const int qB = (b_hi + 1 - boff) * (1 << shift) - 1;
+          const bool open_lo = b_lo == 0, open_hi = b_hi == B - 1;   // the end buckets take whatever falls outside the range
+          // ---- pass 2: gather the hull (raw bits), exact sums of what lies below and above it ----
+          double below = 0.0, above = 0.0;
+          int cnt = 0;
+          for (int c0 = 0; c0 < a.d.C; c0 += 32) {
+            const bool cin = c0 + lane < a.d.C;
+            const float* src = origin + (cin ? c0 + lane : 0) * ch_words;
+            auto sift = [&](float v) {
+              const int q = __float2int_rd(v * qscale);
+              const bool nz = cin && v != 0.0f;
+              const bool lowq = nz && q < qA && !open_lo, highq = nz && q > qB && !open_hi;
+              const bool in = nz && !lowq && !highq;
+              const double dv = (double)v;
+              below = __dadd_rn(below, lowq ? dv : 0.0);
+              above = __dadd_rn(above, highq ? dv : 0.0);
+              const unsigned bal = __ballot_sync(0xFFFFFFFFu, in);
+              if (in) scratch[min(cnt + __popc(bal & lt), kHistCap - 1)] = __float_as_uint(v);
+              cnt += __popc(bal);
+            };
+            if (KHW) {
+#pragma unroll
+              for (int rs = 0; rs < KMAX; ++rs) sift(src[wofs[rs]]);
+            } else {
+              for (int rs = 0; rs < khw; ++rs) sift(src[win[rs]]);
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            below = __dadd_rn(below, __shfl_xor_sync(0xFFFFFFFFu, below, o));
+            above = __dadd_rn(above, __shfl_xor_sync(0xFFFFFFFFu, above, o));
+          }
+          __syncwarp();
+          if (cnt != m_sub) {
+            retry = true;                                            // cannot happen; never trust a mismatch
+          } else {
+            const SplitBase base{s_below, below, above};
+            if (m_sub <= 64) res = hist_sort_select<2>(scratch, m_sub, z_in, a.n, lane, rcp, base);
+            else if (m_sub <= 128) res = hist_sort_select<4>(scratch, m_sub, z_in, a.n, lane, rcp, base);
+            else res = hist_sort_select<8>(scratch, m_sub, z_in, a.n, lane, rcp, base);
+            res.K = __shfl_sync(0xFFFFFFFFu, res.K, 0);
+            res.alpha = __shfl_sync(0xFFFFFFFFu, res.alpha, 0);
+            res.beta = __shfl_sync(0xFFFFFFFFu, res.beta, 0);
+            res.flags = 0u;
+            res.tkey = __shfl_sync(0xFFFFFFFFu, res.tkey, 0);
+            res.mode = __shfl_sync(0xFFFFFFFFu, res.mode, 0);
+            if (res.tkey == kPadKey) retry = true;                   // a split at the hull's outer edge won: not certified
+          }
+          __syncwarp();
+        }
+      }
+      if (retry) {
+        if (lane == 0) ht.retry = 1;
+        continue;
+      }
+      // ---- pass 3: outputs (mask bits in element order, through the offset table) ----
+      if (lane == 0) {
+        a.pK[pi] = res.K;
+        a.pgamma[pi] = res.alpha;
+        a.pdelta[pi] = res.beta;
+        if (a.pflags) a.pflags[pi] = res.flags;
+      }
+      const bool flip = res.mode == 1, none = res.mode == 2;
+      const float tv = key_value(res.tkey);
+      uint32_t mine = 0;
+#pragma unroll 6
+      for (int k = 0; k < rounds; ++k) {
+        const int i = k * 32 + lane;
+        const bool live = i < a.n;
+        const float v = origin[live ? off[i] : 0];
+        const bool bit = !none && live && ((v >= tv) != flip);
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
+        if ((k & 31) == lane) mine = word;
+        if ((k & 31) == 31 || k == rounds - 1) {
+          const int w = (k & ~31) + lane;
+          if (w <= k) mrow[w] = mine;
+        }
+      }
+      for (int w = rounds + lane; w < a.ldp; w += 32) mrow[w] = 0u;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && ht.retry) a.pK[first_patch] = kDenseMark;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Sign coding (the paper's XNOR-structured FBin inputs): mask bit = [x >= 0], gamma = mean |x|, delta = -gamma.
 // One warp per row; `value(i)` returns element i.  HBM-bound work: no sort, one pass.
 // ---------------------------------------------------------------------------------------------------------
@@ -289,6 +658,11 @@ cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64
   return cudaGetLastError();
 }
 
+// 0: sort-based coders (default), 1: histogram-pruned coder where it applies.
+static int g_patch_coder_mode = 0;
+int patch_coder_mode() { return g_patch_coder_mode; }
+void set_patch_coder_mode(int mode) { g_patch_coder_mode = mode; }
+
 // Tile shapes tried, largest first.
 static const int kTileShapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
 
@@ -310,7 +684,7 @@ static void set_tile(const dab_conv_desc& d, int Ho, int Wo, const int (&sh)[2],
 // CTA busy (most CTAs, shortest critical path).  If nothing is admissible the shape with the most resident CTAs wins.
 template <typename Kernel>
 static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes, int threads, int groups,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, bool shape_only = false) {
   const size_t sm_bytes = 228 * 1024, cta_reserve = 1024, cta_limit = 227 * 1024;
   // resident warps per SM a shape must leave room for: measured best is 24 for one or two warps per patch (their
   // tile loads overlap other CTAs' sorting), 16 for larger groups (fewer, larger tiles matter more)
@@ -342,6 +716,7 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
   if (best < 0) return cudaErrorInvalidValue;
   a.tile_shape = best;
   set_tile(a.d, a.Ho, a.Wo, kTileShapes[best], &a);
+  if (shape_only) return cudaSuccess;  // the caller wanted the tile this kernel would take
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)best_smem);
   if (e != cudaSuccess) return e;
   int64_t tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
@@ -357,12 +732,39 @@ static cudaError_t launch_patches_warp(PatchArgs& a, cudaStream_t stream) {
 }
 
 template <int W, int WARPS, int R, bool kFull, bool kTable>
-static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream) {
+static cudaError_t launch_patches_group(PatchArgs& a, cudaStream_t stream, bool shape_only = false) {
   constexpr int G = WARPS / W;
   a.scratch_words = scratch_words_for(a.n, W);
   size_t fixed = (kTable ? sizeof(double) * rcp_table_slots(a.n) : 0) + sizeof(GroupShared) * G +
                  sizeof(uint32_t) * (size_t)a.scratch_words * G;
-  return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, G, stream);
+  return launch_patches(binarize_patches_group_kernel<W, WARPS, R, kFull, kTable>, a, fixed, WARPS * 32, G, stream,
+                        shape_only);
+}
+
+template <int BPL>
+static cudaError_t launch_patches_hist(PatchArgs& a, cudaStream_t stream) {
+  // beyond the group kernel's tile: one more word per channel (odd channel pitch) and the window offsets
+  size_t fixed = sizeof(double) * rcp_table_slots(a.n) + sizeof(int2) * 32 * BPL * kWarpsPerCta +
+                 sizeof(uint32_t) * kHistCap * kWarpsPerCta + sizeof(float) * a.d.C +
+                 sizeof(uint16_t) * (size_t)(a.d.kh * a.d.kw + 2);
+  if (a.d.kh * a.d.kw == 9)
+    return launch_patches(binarize_patches_hist_kernel<BPL, 9>, a, fixed, kWarpsPerCta * 32, kWarpsPerCta, stream);
+  return launch_patches(binarize_patches_hist_kernel<BPL, 0>, a, fixed, kWarpsPerCta * 32, kWarpsPerCta, stream);
+}
+
+// The group kernel that codes patches of n > 256 values (the sort-based coder for these lengths, and the one
+// that takes the tiles the other coders mark).
+static cudaError_t launch_group_for(PatchArgs& a, cudaStream_t stream, bool shape_only) {
+  if (a.n <= 576) return launch_patches_group<4, 8, 5, false, true>(a, stream, shape_only);
+  if (a.n <= 1024) return launch_patches_group<2, 8, 16, false, true>(a, stream, shape_only);
+  if (a.n == 1152) return launch_patches_group<2, 8, 18, true, true>(a, stream, shape_only);
+  if (a.n <= 2048) return launch_patches_group<4, 8, 16, false, true>(a, stream, shape_only);
+  if (a.n == 2304) return launch_patches_group<4, 8, 18, true, true>(a, stream, shape_only);
+  if (a.n <= 4096) return launch_patches_group<8, 16, 16, false, true>(a, stream, shape_only);
+  if (a.n == 4608) return launch_patches_group<8, 16, 18, true, true>(a, stream, shape_only);
+  if (a.n <= 8192) return launch_patches_group<16, 16, 16, false, true>(a, stream, shape_only);
+  if (a.n == 9216) return launch_patches_group<16, 16, 18, true, false>(a, stream, shape_only);
+  return launch_patches_group<16, 16, 32, false, false>(a, stream, shape_only);
 }
 
 cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
@@ -384,11 +786,23 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   a.scratch_words = 0;
   a.defer_dense = 0; a.marked_only = 0; a.tile_shape = -1;
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
-  // The patch lengths of the common 3x3 layers (576 values per warp) have variants without bounds tests whose
-  // group size suits rows that are at least half zeros.  Any other length gets enough warps for at most 16
-  // values per thread, so that rows with up to half their values non-zero sort with 8 keys per thread.
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
-  if (a.n > 256 && a.n <= 576) {
+  if (patch_coder_mode() == 1 && a.n <= 8192) {
+    // Histogram-pruned coder on the tile shape of the group kernel, which then takes the tiles left to it.
+    cudaError_t e = launch_group_for(a, stream, /*shape_only=*/true);
+    if (e != cudaSuccess) return e;
+    if ((size_t)a.d.C * ((a.in_h * a.pitch) | 1) <= 65535) {  // its 16-bit offsets reach the whole (odd-pitched) tile
+      e = a.n < 1024 ? launch_patches_hist<2>(a, stream) : launch_patches_hist<4>(a, stream);
+      if (e != cudaSuccess) return e;
+      a.marked_only = 1;
+    }
+    return launch_group_for(a, stream, false);
+  }
+  // The sort-based coders.  The patch lengths of the common 3x3 layers (576 values per warp) have variants
+  // without bounds tests whose group size suits rows that are at least half zeros.  Any other length gets enough
+  // warps for at most 16 values per thread, so that rows with up to half their values non-zero sort with 8 keys
+  // per thread.
+  if (a.n <= 576) {
     // first the one-warp kernel on the tiles it suits, then four warps per patch on the tiles it marked as dense
     a.defer_dense = 1;
     cudaError_t e = a.n == 576 ? launch_patches_warp<18, true>(a, stream) : launch_patches_warp<18, false>(a, stream);
@@ -396,15 +810,7 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
     a.defer_dense = 0; a.marked_only = 1;  // a.tile_shape now holds the first kernel's tile
     return launch_patches_group<4, 8, 5, false, true>(a, stream);
   }
-  if (a.n <= 1024) return launch_patches_group<2, 8, 16, false, true>(a, stream);
-  if (a.n == 1152) return launch_patches_group<2, 8, 18, true, true>(a, stream);
-  if (a.n <= 2048) return launch_patches_group<4, 8, 16, false, true>(a, stream);
-  if (a.n == 2304) return launch_patches_group<4, 8, 18, true, true>(a, stream);
-  if (a.n <= 4096) return launch_patches_group<8, 16, 16, false, true>(a, stream);
-  if (a.n == 4608) return launch_patches_group<8, 16, 18, true, true>(a, stream);
-  if (a.n <= 8192) return launch_patches_group<16, 16, 16, false, true>(a, stream);
-  if (a.n == 9216) return launch_patches_group<16, 16, 18, true, false>(a, stream);
-  return launch_patches_group<16, 16, 32, false, false>(a, stream);
+  return launch_group_for(a, stream, false);
 }
 
 }  // namespace dab

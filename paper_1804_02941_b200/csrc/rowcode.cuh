@@ -188,9 +188,20 @@ __device__ __forceinline__ RowResult trivial_row(bool bad, float value) {
 // 1e-13 of the maximum are the contenders.  One contender (the usual case) wins outright; several are
 // re-evaluated with the exactly rounded expression and compared as (D, s).  Without the table every split is
 // evaluated exactly.
-template <int W, int E, bool kTable>
+//
+// SplitBase: the keys in r[] may be a contiguous run of the row's sorted order instead of all of it; then s_below
+// elements with sum P_below precede them and elements with sum P_above follow (m, z, and the zero run refer to
+// the run; n to the whole row).  The split before the first key of the run is not evaluated.
+struct SplitBase {
+  int s_below;
+  double P_below, P_above;
+};
+
+template <int W, int E, bool kTable, bool kBased = false>
 __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m, int z, int n, int tig,
-                                                  GroupShared* gs, int bar_id, const double* rcp) {
+                                                  GroupShared* gs, int bar_id, const double* rcp,
+                                                  const SplitBase base = SplitBase{0, 0.0, 0.0}) {
+  const int sb = kBased ? base.s_below : 0;
   constexpr int GT = 32 * W;
   constexpr bool kKeep = kTable && (E <= 8);  // keep fp64 values and fast objectives of this thread in registers
   const int lane = tig & 31, warp = tig >> 5;
@@ -238,6 +249,10 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
     T = __shfl_sync(0xFFFFFFFFu, incl, 31);
     if (lane == 31) next_first = kPadKey;
   }
+  if (kBased) {
+    T = __dadd_rn(__dadd_rn(base.P_below, T), base.P_above);
+    before = __dadd_rn(before, base.P_below);
+  }
   double excl = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
   if (lane == 0) excl = 0.0;
   const double P0 = __dadd_rn(before, excl);  // sum of everything sorted before this thread's keys
@@ -261,14 +276,14 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
       const int q = q0 + j;
       const double P = __dadd_rn(P0, loc[kKeep ? j : 0]);
       if (q + 1 == neg) Pz = P;  // sum of the negatives (P0 itself when neg == q0)
-      const int s = q + 1 + (q >= neg ? z : 0);
+      const int s = sb + q + 1 + (q >= neg ? z : 0);
       const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
       const bool ok = (q < m) && (s < n) && (r[j] != kn);
       double D = ok ? objective_fast(P, T, s, n, rcp) : -1.0;
       Dj[kKeep ? j : 0] = D;
       lmax = fmax(lmax, D);
     }
-    const double Dz = owns_zero_split ? objective_fast(Pz, T, neg + z, n, rcp) : -1.0;
+    const double Dz = owns_zero_split ? objective_fast(Pz, T, sb + neg + z, n, rcp) : -1.0;
     lmax = fmax(lmax, Dz);
     // maximum over the group (lmax >= 0: its bit pattern orders like an integer)
     long long b = __double_as_longlong(lmax);
@@ -304,7 +319,7 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
       uint32_t tk;
       if (j == E) {
         Pc = Pz;
-        s = neg + z;
+        s = sb + neg + z;
         tk = kPadKey;
 #pragma unroll
         for (int i = 0; i < E; ++i)
@@ -319,7 +334,7 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
         }
         Pc = __dadd_rn(P0, lj);
         const int q = q0 + j;
-        s = q + 1 + (q >= neg ? z : 0);
+        s = sb + q + 1 + (q >= neg ? z : 0);
         if (q == neg - 1 && z > 0) tk = kZeroKey;  // the zeros are the smallest values of the high side
       }
       const double D = several ? objective(Pc, T, s, n) : 1.0;
@@ -335,9 +350,9 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
         if (q < m) {
           const uint32_t kc = r[j];
           const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
-          if (q == neg && owns_zero_split) lmax = fmax(lmax, objective_fast(P, T, neg + z, n, rcp));
+          if (q == neg && owns_zero_split) lmax = fmax(lmax, objective_fast(P, T, sb + neg + z, n, rcp));
           P = __dadd_rn(P, (double)key_value(kc));
-          const int s = q + 1 + (q >= neg ? z : 0);
+          const int s = sb + q + 1 + (q >= neg ? z : 0);
           if (s < n && kc != kn) lmax = fmax(lmax, objective_fast(P, T, s, n, rcp));
         }
       }
@@ -364,14 +379,14 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
         const uint32_t kc = r[j];
         const uint32_t kn = (j + 1 < E) ? r[(j + 1 < E) ? j + 1 : j] : next_first;
         if (q == neg && owns_zero_split) {
-          const int s = neg + z;
+          const int s = sb + neg + z;
           if (!kTable || objective_fast(P, T, s, n, rcp) >= thr) {
             double D = objective(P, T, s, n);
             if (D >= bD) { bD = D; bP = P; bS = s; bT = kc; }
           }
         }
         P = __dadd_rn(P, (double)key_value(kc));
-        const int s = q + 1 + (q >= neg ? z : 0);
+        const int s = sb + q + 1 + (q >= neg ? z : 0);
         if (s < n && kc != kn) {
           if (!kTable || objective_fast(P, T, s, n, rcp) >= thr) {
             double D = objective(P, T, s, n);

@@ -1,0 +1,97 @@
+"""The two patch coders (full sort, histogram-pruned search) must give the same codes bit for bit, and the
+histogram coder must match the CPU checker on its own."""
+import numpy as np
+import pytest
+import torch
+
+import dab_synth
+import oracle
+from parity_util import NEAR_TIE, to_dev, unpack, words
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dab():
+    import paper_1804_02941_b200 as d
+    d.lib()
+    oracle.set_threads(8)
+    yield d
+    d.dab_set_patch_coder(d.PATCHES_SORT)
+
+
+def _code(dab, x, C, kh, kw, stride, pad, coder):
+    dab.dab_set_patch_coder(coder)
+    desc = dab.make_desc(tuple(x.shape), 8, kh, kw, stride, pad)
+    Ho, Wo = dab.dab_conv_output_size(desc)
+    P, n = x.shape[0] * Ho * Wo, C * kh * kw
+    ld = dab.dab_default_ld(n)
+    dev = x.device
+    pK = torch.full((P,), -7, dtype=torch.int32, device=dev)
+    pg, pd = torch.zeros(P, device=dev), torch.zeros(P, device=dev)
+    pm = torch.zeros((P, ld), dtype=torch.int32, device=dev)
+    pf = torch.zeros(P, dtype=torch.int32, device=dev)
+    dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, pf)
+    torch.cuda.synchronize()
+    dab.dab_set_patch_coder(dab.PATCHES_SORT)
+    return pK, pg, pd, pm, pf
+
+
+CASES = [
+    # N, C, H, W, kh, kw, stride, pad, kind
+    (2, 64, 20, 20, 3, 3, (1, 1), (1, 1), "relu"),        # n = 576
+    (2, 64, 21, 21, 3, 3, (2, 2), (1, 1), "relu"),
+    (1, 128, 14, 14, 3, 3, (1, 1), (1, 1), "relu"),       # n = 1152
+    (1, 256, 9, 9, 3, 3, (1, 1), (1, 1), "relu"),         # n = 2304
+    (1, 512, 7, 7, 3, 3, (1, 1), (1, 1), "relu"),         # n = 4608
+    (2, 64, 12, 12, 3, 3, (1, 1), (1, 1), "normal"),      # both signs, no zeros
+    (2, 40, 11, 13, 5, 5, (1, 1), (2, 2), "relu"),        # 5x5 window (general path), n = 1000
+    (1, 70, 9, 9, 3, 3, (1, 1), (0, 0), "sparse"),        # 95 % zeros, C not a multiple of 32
+    (1, 64, 10, 10, 3, 3, (1, 1), (1, 1), "negative"),    # no positive value
+    (1, 64, 10, 10, 3, 3, (1, 1), (1, 1), "ints"),        # few distinct values: exact ties, constant patches
+]
+
+
+def _input(kind, shape, stream):
+    if kind == "relu":
+        return dab_synth.relu_activations(shape, 0.6, stream=stream)
+    if kind == "normal":
+        return dab_synth.normal(shape, 1.0, stream=stream)
+    if kind == "sparse":
+        return dab_synth.relu_activations(shape, 0.95, stream=stream)
+    if kind == "negative":
+        return -dab_synth.relu_activations(shape, 0.5, stream=stream)
+    x = np.round(dab_synth.normal(shape, 1.2, stream=stream))
+    x[:, :, :4, :4] = 2.0                                   # constant non-zero patches
+    return x
+
+
+@pytest.mark.parametrize("ci", range(len(CASES)))
+def test_histogram_coder_equals_sort_coder_and_checker(dab, ci):
+    N, C, H, W, kh, kw, stride, pad, kind = CASES[ci]
+    x = _input(kind, (N, C, H, W), 950 + ci).astype(np.float32)
+    xd = to_dev(x)
+    a = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_SORT)
+    b = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_HIST)
+    for s, h in zip(a, b):
+        assert torch.equal(s, h)
+    n = C * kh * kw
+    rows = oracle.im2col(x, kh, kw, stride, pad)
+    sel = np.unique(np.concatenate([[0, len(rows) - 1], (dab_synth.uniform01(96, ci, 0, 64) * len(rows)).astype(np.int64)]))
+    ref = oracle.binarize(rows[sel])
+    strict = ~((ref.gap > 0) & (ref.gap < NEAR_TIE))
+    t = torch.from_numpy(sel).to(xd.device)
+    assert np.array_equal(b[0][t].cpu().numpy()[strict], ref.K[strict])
+    assert np.array_equal(unpack(words(b[3][t]), n)[strict], ref.e[strict])
+    assert np.array_equal(b[4][t].cpu().numpy().view(np.uint32)[strict], ref.flags[strict])
+
+
+def test_nonfinite_tiles_fall_back(dab):
+    x = dab_synth.relu_activations((1, 64, 12, 12), 0.6, stream=990).astype(np.float32)
+    x[0, 3, 5, 5] = np.nan
+    x[0, 9, 0, 11] = np.inf
+    xd = to_dev(x)
+    a = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
+    b = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_HIST)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[3], b[3]) and torch.equal(a[4], b[4])
+    assert int((b[4] == 2).sum()) == 9 + 4
