@@ -10,8 +10,8 @@
 // accumulators per output in tensor memory; M1 = a3 2^24 + a2 2^16 + a1 2^8 + a0 (times 2^-sexp).  The only
 // error is the rounding of x_i to q_i: at most 2^-32 of the row's largest magnitude per element.
 //
-// A CTA owns a tile of TH x TW output positions of one image (at most 128 = the lanes of tensor memory) and 64
-// filters.  It never forms patches in global memory: for each group of 128 patch elements it stages the
+// A CTA owns a tile of TH x TW output positions of one image (at most 128 = the lanes of tensor memory; of
+// several images when a whole image is smaller than that) and 64 filters.  It never forms patches in global memory: for each group of 128 patch elements it stages the
 // channels they come from in shared memory, and every thread gathers 16 consecutive elements of its row,
 // converts them and stores one 16-byte K chunk per byte plane in the operand layout of tc.cuh.
 #include <algorithm>
@@ -39,7 +39,7 @@ constexpr uint32_t WB_BSTAGE = WB_NT * WB_KS;    // bytes of the filter stage
 struct WbinArgs {
   dab_conv_desc d;
   int32_t Ho, Wo, n, words, khw;
-  int32_t TH, TW, tiles_h, tiles_w;
+  int32_t TH, TW, TI, tiles_h, tiles_w;  // tile: TI images x TH x TW output positions (TI > 1 only when one tile covers an image)
   int32_t in_h, in_w, pitch, ch_words, max_ch;
   uint32_t magic_npix, magic_in_w, magic_khw, magic_kw;  // ceil(2^32 / d): floor(i / d) = umulhi(i, magic); 0 if d == 1
   const float* x;
@@ -114,18 +114,21 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
   unsigned char* const stage_a = dyn_mem + (mem0 - smem_u32(dyn_mem));
   unsigned char* const stage_b = stage_a + 4 * WB_PLANE;
   // two input tiles: the next group of channels arrives while the current one is gathered
-  const int tile_words = a.max_ch * a.ch_words;
+  const int img_words = a.max_ch * a.ch_words;  // staged words of one image of the tile
+  const int tile_words = a.TI * img_words;
   float* const tiles = reinterpret_cast<float*>(stage_b + WB_BSTAGE);
   uint32_t* const pixmax = reinterpret_cast<uint32_t*>(tiles + 2 * (size_t)tile_words);
   const uint32_t bar = smem_u32(&s_bar);
 
   // tile of this CTA
   const int tiles_per_img = a.tiles_h * a.tiles_w;
-  const int img = blockIdx.x / tiles_per_img, trem = blockIdx.x % tiles_per_img;
+  const int img0 = (blockIdx.x / tiles_per_img) * a.TI, trem = blockIdx.x % tiles_per_img;
+  const int imgs = min(a.TI, a.d.N - img0);  // images of this tile
   const int ho0 = (trem / a.tiles_w) * a.TH, wo0 = (trem % a.tiles_w) * a.TW;
   const int h0 = ho0 * a.d.stride_h - a.d.pad_h, w0 = wo0 * a.d.stride_w - a.d.pad_w;
   const int j0 = blockIdx.y * WB_NT;
-  const float* const ximg = a.x + (int64_t)img * a.d.C * a.d.H * a.d.W;
+  const int64_t img_stride = (int64_t)a.d.C * a.d.H * a.d.W;
+  const float* const x0 = a.x + (int64_t)img0 * img_stride;
   const int npix = a.in_h * a.in_w;
 
   if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 4 * WB_NT);
@@ -139,28 +142,31 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
     s_beta[j] = in ? (double)a.wbeta[j0 + j] : 0.0;
   }
   // per-pixel maxima of the staged region (0 outside the image)
-  for (int pix = tid; pix < npix; pix += WB_THREADS) {
+  for (int idx = tid; idx < imgs * npix; idx += WB_THREADS) {
+    const int ti = fast_div(idx, a.magic_npix), pix = idx - ti * npix;
     const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
     const int h = h0 + r, w = w0 + s;
     uint32_t m = 0u;
     if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
-      m = __ldg(a.pixmax + ((int64_t)img * a.d.H + h) * a.d.W + w);
-    pixmax[pix] = m;
+      m = __ldg(a.pixmax + ((int64_t)(img0 + ti) * a.d.H + h) * a.d.W + w);
+    pixmax[idx] = m;
   }
   __syncthreads();
 
   // Row = output position (lh, lw) of the tile; its scale comes from the largest magnitude of its patch.
   const int row = tid & (kLanes - 1), half = tid >> 7;
-  const int lh = row / a.TW, lw = row - lh * a.TW;
-  const bool row_in = lh < a.TH && ho0 + lh < a.Ho && wo0 + lw < a.Wo;
-  const int origin = lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
+  const int per_img = a.TH * a.TW;
+  const int rti = row / per_img, rrem = row - rti * per_img;  // image of the tile, position inside it
+  const int lh = rrem / a.TW, lw = rrem - lh * a.TW;
+  const bool row_in = rti < imgs && ho0 + lh < a.Ho && wo0 + lw < a.Wo;
+  const int origin = rti * img_words + lh * a.d.stride_h * a.pitch + lw * a.d.stride_w;
   if (tid < kLanes) {
     int sexp = INT_MIN;
     if (row_in) {
       uint32_t m = 0u;
       for (int i = 0; i < a.d.kh; ++i)
         for (int j = 0; j < a.d.kw; ++j)
-          m = max(m, pixmax[(lh * a.d.stride_h + i) * a.in_w + lw * a.d.stride_w + j]);
+          m = max(m, pixmax[rti * npix + (lh * a.d.stride_h + i) * a.in_w + lw * a.d.stride_w + j]);
       if (m >= 0x7F800000u) sexp = INT_MAX;
       else if (m == 0u) sexp = 0;
       else sexp = 30 - ((int)(m >> 23) - 127);  // -97 .. 157 (the largest for a subnormal maximum)
@@ -187,16 +193,19 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
   auto stage_in = [&](int st) {
     const int k0 = st * WB_KS, k1 = min(a.n, k0 + WB_KS);
     const int c_lo = fast_div(k0, a.magic_khw), c_hi = fast_div(k1 - 1, a.magic_khw) + 1;
-    float* const tile = tiles + (st & 1) * tile_words;
-    for (int idx = tid; idx < (c_hi - c_lo) * npix; idx += WB_THREADS) {
-      const int c = fast_div(idx, a.magic_npix), pix = idx - c * npix;
-      const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
-      const int h = h0 + r, w = w0 + s;
-      const bool in = (unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W;
-      const float* src = in ? ximg + ((int64_t)(c_lo + c) * a.d.H + h) * a.d.W + w : ximg;
-      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(tile + c * a.ch_words + r * a.pitch + s)),
-                   "l"(src), "r"(in ? 4 : 0)
-                   : "memory");  // source size 0: the word is filled with zeros
+    for (int ti = 0; ti < imgs; ++ti) {
+      float* const tile = tiles + (st & 1) * tile_words + ti * img_words;
+      const float* const ximg = x0 + ti * img_stride;
+      for (int idx = tid; idx < (c_hi - c_lo) * npix; idx += WB_THREADS) {
+        const int c = fast_div(idx, a.magic_npix), pix = idx - c * npix;
+        const int r = fast_div(pix, a.magic_in_w), s = pix - r * a.in_w;
+        const int h = h0 + r, w = w0 + s;
+        const bool in = (unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W;
+        const float* src = in ? ximg + ((int64_t)(c_lo + c) * a.d.H + h) * a.d.W + w : ximg;
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(tile + c * a.ch_words + r * a.pitch + s)),
+                     "l"(src), "r"(in ? 4 : 0)
+                     : "memory");  // source size 0: the word is filled with zeros
+      }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
     if (tid < WB_KS) {
@@ -277,7 +286,8 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
   // Epilogue: thread = row (a warp reads the 32 lanes of its quarter), warps 0-3 the first 32 filters, 4-7 the rest.
   {
     const int erow = (warp & 3) * 32 + lane;
-    const int elh = erow / a.TW, elw = erow - elh * a.TW;
+    const int eti = erow / per_img, erem = erow - eti * per_img;
+    const int elh = erem / a.TW, elw = erem - elh * a.TW;
     const int sexp = s_rowsexp[erow];
     const bool valid = sexp != INT_MIN && !dead;
     const bool bad = sexp == INT_MAX;
@@ -292,7 +302,7 @@ __global__ void __launch_bounds__(WB_THREADS, 2) wbin_conv_kernel(const WbinArgs
     }
     const double Sd = (double)S;
     const int64_t plane_hw = (int64_t)a.Ho * a.Wo;
-    const int64_t obase = (int64_t)img * a.d.Cout * plane_hw + (int64_t)(ho0 + elh) * a.Wo + (wo0 + elw);
+    const int64_t obase = (int64_t)(img0 + eti) * a.d.Cout * plane_hw + (int64_t)(ho0 + elh) * a.Wo + (wo0 + elw);
     const int cb = warp >> 2;
 #pragma unroll 1
     for (int c8 = 0; c8 < 4; ++c8) {
@@ -383,11 +393,21 @@ cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, con
   if (smem > limit1 || (size_t)a.max_ch * a.ch_words > 65535) return cudaErrorInvalidValue;
   a.tiles_h = (Ho + a.TH - 1) / a.TH;
   a.tiles_w = (Wo + a.TW - 1) / a.TW;
+  // Small images (one tile each, e.g. fully connected layers as 1x1 outputs): a tile takes as many images as
+  // fit the 128 lanes and shared memory, so that the expansion of the filter masks is shared by more rows.
+  a.TI = 1;
+  if (a.tiles_h == 1 && a.tiles_w == 1) {
+    const size_t per_img = 2 * sizeof(float) * (size_t)a.max_ch * a.ch_words + sizeof(uint32_t) * (size_t)a.in_h * a.in_w;
+    int ti = std::min<int64_t>(d.N, kLanes / (a.TH * a.TW));
+    while (ti > 1 && fixed + ti * per_img > limit1) --ti;
+    a.TI = ti;
+    smem = fixed + ti * per_img;
+  }
   a.magic_npix = magic_for((uint32_t)(a.in_h * a.in_w));
   a.magic_in_w = magic_for((uint32_t)a.in_w);
   a.magic_khw = magic_for((uint32_t)a.khw);
   a.magic_kw = magic_for((uint32_t)d.kw);
-  const int64_t gx = (int64_t)d.N * a.tiles_h * a.tiles_w;
+  const int64_t gx = (int64_t)((d.N + a.TI - 1) / a.TI) * a.tiles_h * a.tiles_w;
   const int64_t gy = (d.Cout + WB_NT - 1) / WB_NT;
   if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
   const int64_t HW = (int64_t)d.H * d.W, pixels = (int64_t)d.N * HW;
