@@ -374,17 +374,19 @@ def run_dab(args):
     e2e = None
     if not args.no_e2e:
         max_ws = max(dab.dab_binary_conv_host_workspace(desc) for (_, _, _, _, desc, _, _) in work)
-        ws = torch.empty(max_ws, dtype=torch.uint8, device=dev)
-        y_host = torch.empty(max_y, dtype=torch.float32).pin_memory()
+        # two workspaces, taken in turn: a layer is queued while the one before it is still copying out
+        wss = [torch.empty(max_ws, dtype=torch.uint8, device=dev) for _ in range(2)]
+        y_hosts = [torch.empty(max_y, dtype=torch.float32).pin_memory() for _ in range(2)]
         h2d = sum(4 * L.N * L.C * L.H * L.W for L in layers)
         d2h = sum(4 * L.patches * L.Cout for L in layers)
 
         def e2e_step():
-            for (L, x, w, wc, desc, pm, y) in work:
+            for li, (L, x, w, wc, desc, pm, y) in enumerate(work):
                 dab.dab_binarize_into(w, wc.K, wc.alpha, wc.beta, wc.mask, wc.flags, stream=stream)
-                yh = y_host[: L.patches * L.Cout].view(L.N, L.Cout, L.Ho, L.Wo)
+                yh = y_hosts[li & 1][: L.patches * L.Cout].view(L.N, L.Cout, L.Ho, L.Wo)
                 dab.dab_binary_conv_host(host_x[L.x_shape()], wc, L.kh, L.kw, (L.stride, L.stride), (L.pad, L.pad),
-                                         y_host=yh, workspace=ws, stream=stream)
+                                         y_host=yh, workspace=wss[li & 1], stream=stream, wait=False)
+            dab.dab_binary_conv_host_wait(stream)
         e2e_step()
         barrier()
         torch.cuda.synchronize()

@@ -232,6 +232,20 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
                                 void* d_workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * dab_binary_conv_host_async — the same call without the final wait: it returns once all its copies and kernels
+ * are queued, so that the next layer's copy-in overlaps this layer's last kernels and copy-out.  h_y is complete,
+ * and h_x, the filters and the workspace may be reused or freed, only after dab_binary_conv_host_wait (or a later
+ * dab_binary_conv_host on the device) has returned.  A call whose workspace overlaps that of one of the last two
+ * unfinished calls waits for it on the device, and at most two calls are left running at a time: give
+ * consecutive layers two alternating workspaces to let them overlap.
+ * dab_binary_conv_host_wait — blocks until every such call on the current device, and `stream`, have finished.
+ */
+dab_status dab_binary_conv_host_async(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask,
+                                      int32_t ldw, const int32_t* d_wK, const float* d_walpha, const float* d_wbeta,
+                                      float* h_y, void* d_workspace, size_t workspace_bytes, void* stream);
+dab_status dab_binary_conv_host_wait(void* stream);
+
+/*
  * dab_binary_conv_static — dab_binary_conv without a workspace argument.  The paper has no counterpart: this
  * entry point exists for callers that cannot allocate device memory themselves, for example code running
  * inside a plugin or callback interface that hands it device pointers for inputs and outputs only, or a

@@ -24,7 +24,7 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
-           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward", "dab_set_patch_coder", "dab_get_patch_coder")
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward", "dab_set_patch_coder", "dab_get_patch_coder", "dab_binary_conv_host_async", "dab_binary_conv_host_wait")
 
 
 class DabError(RuntimeError):
@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_sign.argtypes = L.dab_binary_conv.argtypes
         L.dab_binary_conv_contract.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.dab_binary_conv_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.dab_binary_conv_host_async.argtypes = L.dab_binary_conv_host.argtypes
+        L.dab_binary_conv_host_wait.argtypes = [vp]
         L.dab_binary_conv_static_capacity.restype = C.c_size_t
         L.dab_binary_conv_static_capacity.argtypes = []
         L.dab_binary_conv_static.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
@@ -284,8 +286,10 @@ def dab_binary_conv_contract(desc: ConvDesc, pmask, pK, pgamma, pdelta, w: Coded
 
 
 def dab_binary_conv_host(x_host: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
-                         y_host: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None):
-    """Host tensors in and out (pinned memory recommended); the library does the copies. Synchronous."""
+                         y_host: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None,
+                         wait: bool = True):
+    """Host tensors in and out (pinned memory recommended); the library does the copies.  wait=False queues the
+    layer and returns (dab_binary_conv_host_async): call dab_binary_conv_host_wait before reading y_host."""
     if x_host.is_cuda or x_host.dtype != torch.float32 or not x_host.is_contiguous():
         raise TypeError("x_host must be a contiguous fp32 host tensor")
     Cout = w.mask.shape[0]
@@ -295,12 +299,20 @@ def dab_binary_conv_host(x_host: torch.Tensor, w: Coded, kh: int, kw: int, strid
         y_host = torch.empty((x_host.shape[0], Cout, Ho, Wo), dtype=torch.float32).pin_memory()
     need = dab_binary_conv_host_workspace(desc)
     if workspace is None:
+        if not wait:
+            raise ValueError("wait=False needs a caller-owned workspace that outlives the queued work")
         workspace = torch.empty(need, dtype=torch.uint8, device=w.mask.device)
-    st = lib().dab_binary_conv_host(C.byref(desc), C.c_void_p(x_host.data_ptr()), _ptr(w.mask), w.ld, _ptr(w.K),
+    fn = lib().dab_binary_conv_host if wait else lib().dab_binary_conv_host_async
+    st = fn(C.byref(desc), C.c_void_p(x_host.data_ptr()), _ptr(w.mask), w.ld, _ptr(w.K),
                                     _ptr(w.alpha), _ptr(w.beta), C.c_void_p(y_host.data_ptr()), _ptr(workspace),
                                     workspace.numel(), _stream(stream))
     _check(st, "dab_binary_conv_host")
     return y_host
+
+
+def dab_binary_conv_host_wait(stream=None) -> None:
+    """Blocks until every layer queued with wait=False on the current device has finished."""
+    _check(lib().dab_binary_conv_host_wait(_stream(stream)), "dab_binary_conv_host_wait")
 
 
 def dab_binary_conv_static_capacity() -> int:

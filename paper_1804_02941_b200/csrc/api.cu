@@ -259,6 +259,15 @@ struct HostPipe {
   bool ready = false;
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t start = nullptr, in_done[2] = {}, comp_done[2] = {}, out_done[2] = {};
+  // The last two calls that were left running (dab_binary_conv_host_async): their workspace ranges and the events
+  // that mark the end of their kernels and of their copies out.  A new call waits for those whose workspace it touches.
+  struct Tail {
+    const char* lo = nullptr;
+    const char* hi = nullptr;
+    cudaEvent_t comp = nullptr, out = nullptr;
+    bool live = false;
+  } tail[2];
+  int next_tail = 0;
 };
 
 std::mutex g_host_mutex;
@@ -278,6 +287,8 @@ cudaError_t host_pipe(HostPipe** out) {
       if ((e = cudaEventCreateWithFlags(&p.in_done[b], cudaEventDisableTiming)) != cudaSuccess) return e;
       if ((e = cudaEventCreateWithFlags(&p.comp_done[b], cudaEventDisableTiming)) != cudaSuccess) return e;
       if ((e = cudaEventCreateWithFlags(&p.out_done[b], cudaEventDisableTiming)) != cudaSuccess) return e;
+      if ((e = cudaEventCreateWithFlags(&p.tail[b].comp, cudaEventDisableTiming)) != cudaSuccess) return e;
+      if ((e = cudaEventCreateWithFlags(&p.tail[b].out, cudaEventDisableTiming)) != cudaSuccess) return e;
     }
     p.ready = true;
   }
@@ -316,9 +327,9 @@ size_t dab_binary_conv_host_workspace(const dab_conv_desc* desc) {
   return p.total;
 }
 
-dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,
-                                const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* h_y,
-                                void* d_workspace, size_t workspace_bytes, void* stream) {
+static dab_status conv_host(bool drain, const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,
+                            const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* h_y,
+                            void* d_workspace, size_t workspace_bytes, void* stream) {
   ConvGeom g;
   HostPlan pl;
   if (!conv_geom(desc, &g) || !host_plan(desc, g, &pl)) return DAB_ERR_INVALID_ARG;
@@ -338,6 +349,20 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
                            cudaStreamSynchronize(st); return DAB_ERR_CUDA; } } while (0)
   DAB_TRY(cudaEventRecord(hp->start, st));  // work already queued on the caller's stream comes first
   DAB_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+  // earlier calls still running on a workspace that overlaps this one (or about to lose their record) come first
+  HostPipe::Tail& slot = hp->tail[hp->next_tail];
+  for (int i = 0; i < 2; ++i) {
+    HostPipe::Tail& t = hp->tail[i];
+    if (!t.live) continue;
+    const bool overlap = ws < t.hi && t.lo < ws + pl.total;
+    if (overlap || &t == &slot) {
+      DAB_TRY(cudaStreamWaitEvent(hp->in, t.comp, 0));
+      DAB_TRY(cudaStreamWaitEvent(hp->in, t.out, 0));
+      DAB_TRY(cudaStreamWaitEvent(st, t.comp, 0));
+      DAB_TRY(cudaStreamWaitEvent(st, t.out, 0));
+      if (&t == &slot) t.live = false;
+    }
+  }
   dab_status status = DAB_OK;
   for (int c = 0; c < pl.chunks; ++c) {
     const int b = c & 1;
@@ -363,9 +388,41 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
                             cudaMemcpyDeviceToHost, hp->out));
     DAB_TRY(cudaEventRecord(hp->out_done[b], hp->out));
   }
+  if (!drain && status == DAB_OK) {  // leave it running: remember what it occupies
+    DAB_TRY(cudaEventRecord(slot.comp, st));
+    DAB_TRY(cudaEventRecord(slot.out, hp->out));
+    slot.lo = ws;
+    slot.hi = ws + pl.total;
+    slot.live = true;
+    hp->next_tail ^= 1;
+    return DAB_OK;
+  }
 #undef DAB_TRY
   cudaError_t e1 = cudaStreamSynchronize(hp->in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(hp->out);
+  hp->tail[0].live = hp->tail[1].live = false;  // the copy-out stream has drained: nothing is left running
   if (status != DAB_OK) return status;
+  return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess) ? DAB_OK : DAB_ERR_CUDA;
+}
+
+dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,
+                                const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* h_y,
+                                void* d_workspace, size_t workspace_bytes, void* stream) {
+  return conv_host(true, desc, h_x, d_wmask, ldw, d_wK, d_walpha, d_wbeta, h_y, d_workspace, workspace_bytes, stream);
+}
+
+dab_status dab_binary_conv_host_async(const dab_conv_desc* desc, const float* h_x, const uint32_t* d_wmask, int32_t ldw,
+                                      const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* h_y,
+                                      void* d_workspace, size_t workspace_bytes, void* stream) {
+  return conv_host(false, desc, h_x, d_wmask, ldw, d_wK, d_walpha, d_wbeta, h_y, d_workspace, workspace_bytes, stream);
+}
+
+dab_status dab_binary_conv_host_wait(void* stream) {
+  std::lock_guard<std::mutex> lock(g_host_mutex);
+  HostPipe* hp = nullptr;
+  if (host_pipe(&hp) != cudaSuccess) return DAB_ERR_CUDA;
+  cudaError_t e1 = cudaStreamSynchronize(hp->in), e2 = cudaStreamSynchronize(static_cast<cudaStream_t>(stream)),
+              e3 = cudaStreamSynchronize(hp->out);
+  hp->tail[0].live = hp->tail[1].live = false;
   return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess) ? DAB_OK : DAB_ERR_CUDA;
 }
 

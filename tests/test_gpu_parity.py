@@ -255,6 +255,30 @@ def test_conv_host_entry_point(dab, batch):
     assert torch.equal(y_pageable, y_dev)
 
 
+def test_conv_host_layers_queued_without_waiting(dab):
+    # five layers queued back to back: alternating workspaces (they may overlap on the device), then one shared
+    # workspace (each call must wait for the one before it); every output equals the device-resident call
+    shapes = [(7, 16, 12, 12, 24), (5, 8, 20, 20, 16), (9, 32, 9, 9, 8), (4, 16, 12, 12, 24), (6, 8, 20, 20, 16)]
+    layers = [configs.ConvLayer("q%d" % i, *sh, 3, 3, 1, 1) for i, sh in enumerate(shapes)]
+    xs = [torch.from_numpy(L.inputs(stream=30 + i)).pin_memory() for i, L in enumerate(layers)]
+    wds = [dab.dab_binarize(to_dev(L.weights(stream=30 + i))) for i, L in enumerate(layers)]
+    refs = [dab.dab_binary_conv(x.cuda(), wd, 3, 3, (1, 1), (1, 1)).cpu() for x, wd in zip(xs, wds)]
+    descs = [dab.make_desc(L.x_shape(), L.Cout, 3, 3, (1, 1), (1, 1)) for L in layers]
+    need = max(dab.dab_binary_conv_host_workspace(d) for d in descs)
+    for n_ws in (2, 1):
+        wss = [torch.empty(need, dtype=torch.uint8, device="cuda") for _ in range(n_ws)]
+        ys = [torch.empty_like(r).pin_memory() for r in refs]
+        for rep in range(2):
+            for i, (x, wd) in enumerate(zip(xs, wds)):
+                dab.dab_binary_conv_host(x, wd, 3, 3, (1, 1), (1, 1), y_host=ys[i], workspace=wss[i % n_ws], wait=False)
+            dab.dab_binary_conv_host_wait()
+            for y, r in zip(ys, refs):
+                assert torch.equal(y, r)
+                y.zero_()
+    with pytest.raises(ValueError):
+        dab.dab_binary_conv_host(xs[0], wds[0], 3, 3, (1, 1), (1, 1), wait=False)
+
+
 def test_argument_errors_are_return_codes(dab):
     import ctypes as C
     L = dab.lib()
