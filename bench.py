@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"],
                     help="contraction kernel: auto (tensor cores except on tiny problems; every layer of this workload takes "
                          "them), tensor (forced) or popc (AND + population counts)")
+    ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist"],
+                    help="patch coder: auto (by tile density), sort (full sort per patch) or hist (histogram-pruned search)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -202,6 +204,17 @@ def run_reference(args):
     }))
 
 
+def patch_launches(n, coder):
+    """Kernels one dab_binarize_patches call launches (some end at once when no tile was handed to them)."""
+    if n <= 256:
+        return 1
+    if coder == "auto":
+        return 3                      # sort-based coder, histogram coder on the dense tiles, group kernel on the rest
+    if coder == "hist":
+        return 2
+    return 2 if n <= 576 else 1       # one warp per patch, then the group kernel on the tiles marked dense
+
+
 def select_layers(layers, args):
     if not args.layers:
         return layers
@@ -218,7 +231,7 @@ def workload_config(args, batch_override=None):
             "workload": "config 5: ResNet-18-shaped stack of 16 binarized 3x3 convolutions (64/128/256/512 channels, "
                         "56/28/14/7 px), per-filter and per-patch distribution-aware binarization, AND-popcount contraction",
             "batch_per_gpu": b, "inputs": "dense N(0,1)" if args.dense else "post-ReLU half-normal, 60% exact zeros",
-            "weights": "N(0, 0.02^2)", "l2": "no flush: a step streams >3 GB of distinct inputs and outputs, L2 is 126 MB",
+            "weights": "N(0, 0.02^2)", "patch_coder": args.patch_coder, "l2": "no flush: a step streams >3 GB of distinct inputs and outputs, L2 is 126 MB",
             "parallelism": "replicas" if args.gpus > 1 else "single GPU"}
 
 
@@ -241,6 +254,7 @@ def run_dab(args):
         dist.init_process_group("nccl", device_id=dev)
     dab.lib()
     dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
+    dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST}[args.patch_coder])
     hbm_peak, peak_src, sm_max_mhz = load_peaks()
 
     layers = select_layers(configs.config5(args.batch), args)
@@ -439,7 +453,7 @@ def run_dab(args):
                "scaling": "weak", "vs_baseline": None, "dtype": "u8 x u8 -> s32 tensor-core counts + f64 objective/rescale" if args.contraction != "popc"
                else "u32 popcount + f64 objective/rescale",
                "data": "synthetic", "config": workload_config(args), "clocks": clocks, "e2e": e2e,
-               "gpu_launches": 3 * launches_per_kind,
+               "gpu_launches": (2 * len(layers) + sum(patch_launches(L.n, args.patch_coder) for L in layers)) * args.steps,
                "kernel_ms_per_step": {k: v / args.steps for k, v in k_ms.items()},
                "binarize_gbs": binarize_gbs, "roofline": roofline, "roofline_contraction": roofline_contract,
                "wbin": wbin, "cpu_baseline": cpu_baseline, "contraction_wait_failures": dab.dab_contraction_wait_failures()}

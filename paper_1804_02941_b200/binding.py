@@ -410,11 +410,11 @@ def dab_set_contraction(path: int) -> None:
     _check(lib().dab_set_contraction(int(path)), "dab_set_contraction")
 
 
-PATCHES_SORT, PATCHES_HIST = 0, 1
+PATCHES_AUTO, PATCHES_SORT, PATCHES_HIST = 0, 1, 2
 
 
 def dab_set_patch_coder(coder: int) -> None:
-    """PATCHES_SORT (default: full sort per patch) or PATCHES_HIST (histogram-pruned search where it applies)."""
+    """PATCHES_AUTO (default: by tile density), PATCHES_SORT (full sort per patch) or PATCHES_HIST (histogram-pruned search)."""
     _check(lib().dab_set_patch_coder(int(coder)), "dab_set_patch_coder")
 
 

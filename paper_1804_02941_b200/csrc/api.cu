@@ -433,12 +433,12 @@ dab_status dab_set_contraction(dab_contraction path) {
 }
 
 dab_status dab_set_patch_coder(dab_patch_coder coder) {
-  if (coder != DAB_PATCHES_SORT && coder != DAB_PATCHES_HIST) return DAB_ERR_INVALID_ARG;
-  set_patch_coder_mode(coder == DAB_PATCHES_HIST ? 1 : 0);
+  if (coder != DAB_PATCHES_AUTO && coder != DAB_PATCHES_SORT && coder != DAB_PATCHES_HIST) return DAB_ERR_INVALID_ARG;
+  set_patch_coder_mode((int)coder);
   return DAB_OK;
 }
 
-dab_patch_coder dab_get_patch_coder(void) { return patch_coder_mode() == 1 ? DAB_PATCHES_HIST : DAB_PATCHES_SORT; }
+dab_patch_coder dab_get_patch_coder(void) { return (dab_patch_coder)patch_coder_mode(); }
 
 dab_contraction dab_get_contraction(void) { return (dab_contraction)g_contraction.load(std::memory_order_relaxed); }
 

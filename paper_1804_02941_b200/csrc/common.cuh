@@ -91,7 +91,7 @@ cudaError_t read_mma_wait_timeouts(unsigned int* count);
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
                                     float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
                                     cudaStream_t stream);
-// Patch coder selection: 0 sort-based (default), 1 histogram-pruned where it applies.
+// Patch coder selection: 0 by tile density (default), 1 sort-based only, 2 histogram-pruned wherever it applies.
 int patch_coder_mode();
 void set_patch_coder_mode(int mode);
 cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K, float* alpha,

@@ -1,5 +1,7 @@
 // The patch coder of dab_binary_conv: the row coder of rowcode.cuh applied to every patch of an NCHW tensor
 // (one warp per patch for up to 1024 values, a group of 2..16 warps beyond).
+#include <atomic>
+
 #include "rowcode.cuh"
 
 namespace dab {
@@ -17,8 +19,15 @@ struct PatchArgs {
   int32_t pitch;           // words per staged row (>= in_w)
   int32_t tiles_h, tiles_w;
   int32_t scratch_words;
-  int32_t defer_dense;     // one-warp kernel: leave tiles that look dense to a second kernel (marks them in pK)
-  int32_t marked_only;     // group kernel: code only the tiles marked by the one-warp kernel
+  int32_t defer_dense;     // leave tiles that look dense to the next kernel of the chain (marks them in pK)
+  int32_t dense_num, dense_den;  // a tile is dense if non-zero staged values * dense_den > staged values * dense_num
+  int32_t marked_only;     // code only the tiles marked by the kernel before
+  // Chains of kernels on one stream hand tiles on through marks.  So that a kernel with nothing to do ends at
+  // once, the kernel that marks a tile also writes the call's id to *flag_out, and a marked-only kernel leaves
+  // at entry unless *flag_in holds that id.  (Either pointer may be null: no flag written / always run.)
+  uint32_t call_id;
+  unsigned int* flag_in;
+  unsigned int* flag_out;
   int32_t tile_shape;      // index into kTileShapes forced by the caller, -1: choose
   uint32_t magic_per_ch, magic_in_w;  // ceil(2^32 / d) for d = in_h*in_w and in_w: floor(i/d) = umulhi(i, magic); 0 if d == 1
   const float* x;
@@ -84,6 +93,24 @@ __device__ __forceinline__ TileCoord tile_coord(const PatchArgs& a, int64_t tile
   return t;
 }
 
+// Staged values of a tile that come from the image (the rest is zero padding): what its density is measured on.
+__device__ __forceinline__ int64_t staged_inside(const PatchArgs& a, const TileCoord& t) {
+  const int rows = min(t.h0 + a.in_h, a.d.H) - max(t.h0, 0), cols = min(t.w0 + a.in_w, a.d.W) - max(t.w0, 0);
+  return (int64_t)a.d.C * max(rows, 0) * max(cols, 0);
+}
+
+// Whether a marked-only kernel has anything to do in this CTA: the call's flag says that some tile was marked at
+// all, then the marks of the CTA's own tiles are read.  Every thread of the CTA gets the same answer.
+__device__ __forceinline__ bool has_marked_tile(const PatchArgs& a) {
+  if (a.flag_in && *reinterpret_cast<volatile unsigned int*>(a.flag_in) != a.call_id) return false;
+  const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
+  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+    const TileCoord t = tile_coord(a, tile_id);
+    if (a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] == kDenseMark) return true;
+  }
+  return false;
+}
+
 #ifndef DAB_WARP_MINBLOCKS
 #define DAB_WARP_MINBLOCKS 3  // CTAs per SM the one-warp-per-patch kernel is compiled for (register budget)
 #endif
@@ -120,9 +147,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
       nz = __reduce_add_sync(0xFFFFFFFFu, nz);
       if (lane == 0 && nz) atomicAdd(&tile_nonzero, nz);
       __syncthreads();
-      const int64_t staged = (int64_t)a.d.C * a.in_h * a.in_w;
-      if ((int64_t)tile_nonzero * a.n > 256 * staged) {
-        if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+      const int64_t staged = staged_inside(a, t);
+      if ((int64_t)tile_nonzero * a.dense_den > a.dense_num * staged) {
+        if (threadIdx.x == 0) {
+          a.pK[first_patch] = kDenseMark;
+          if (a.flag_out) *a.flag_out = a.call_id;
+        }
         continue;
       }
     } else {
@@ -166,16 +196,34 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
   GroupShared* gs = gs_all + group;
   uint32_t* scratch = scratch_all + (size_t)group * a.scratch_words;
   const int bar_id = 1 + group;
+  if (a.marked_only && !has_marked_tile(a)) return;
+  __shared__ int tile_nonzero;
   if (kTable) fill_reciprocals(rcp, a.n, threadIdx.x, THREADS);
   fill_offsets(a, off, ch_words, threadIdx.x, THREADS);
 
   const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
-    if (a.marked_only && a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] != kDenseMark) continue;
+    const int64_t first_patch = ((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0;
+    if (a.marked_only && a.pK[first_patch] != kDenseMark) continue;
     __syncthreads();
-    load_tile<true>(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x, THREADS);
+    if (threadIdx.x == 0) tile_nonzero = 0;
+    int nz = load_tile<true>(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x,
+                             THREADS);
     __syncthreads();
+    if (a.defer_dense) {  // dense tiles go to the next kernel of the chain
+      nz = __reduce_add_sync(0xFFFFFFFFu, nz);
+      if ((threadIdx.x & 31) == 0 && nz) atomicAdd(&tile_nonzero, nz);
+      __syncthreads();
+      const int64_t staged = staged_inside(a, t);
+      if ((int64_t)tile_nonzero * a.dense_den > a.dense_num * staged) {
+        if (threadIdx.x == 0) {
+          a.pK[first_patch] = kDenseMark;
+          if (a.flag_out) *a.flag_out = a.call_id;
+        }
+        continue;
+      }
+    }
 
     for (int p = group; p < t.th * t.tw; p += G) {
       const int lh = p / t.tw, lw = p % t.tw;
@@ -262,6 +310,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
   uint16_t* win = off + ((a.n + 1) & ~1);       // offsets of the kernel window inside one channel
   __shared__ HistTile ht;
 
+  if (a.marked_only && !has_marked_tile(a)) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int2* hist = hist_all + warp * B;
   uint32_t* scratch = scratch_all + warp * kHistCap;
@@ -283,6 +332,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
   const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
+    if (a.marked_only && a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] != kDenseMark) continue;
     __syncthreads();  // the previous tile is no longer read
     if (threadIdx.x == 0) { ht.kmin = kPadKey; ht.kmax = 0u; ht.retry = 0; }
     __syncthreads();
@@ -318,7 +368,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
     const uint32_t tkmin = ht.kmin, tkmax = ht.kmax;
     const bool any_nonzero = tkmin <= tkmax;
     if (any_nonzero && key_range_nonfinite(tkmin, tkmax)) {
-      if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+      if (threadIdx.x == 0) {
+        a.pK[first_patch] = kDenseMark;
+        if (a.flag_out) *a.flag_out = a.call_id;
+      }
       continue;
     }
     // Quantisation of the tile: q = floor(v * qscale); bucket = (q >> shift) + boff; B0 = first bucket of positives.
@@ -562,7 +615,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
       for (int w = rounds + lane; w < a.ldp; w += 32) mrow[w] = 0u;
     }
     __syncthreads();
-    if (threadIdx.x == 0 && ht.retry) a.pK[first_patch] = kDenseMark;
+    if (threadIdx.x == 0 && ht.retry) {
+      a.pK[first_patch] = kDenseMark;
+      if (a.flag_out) *a.flag_out = a.call_id;
+    }
   }
 }
 
@@ -658,8 +714,32 @@ cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64
   return cudaGetLastError();
 }
 
-// 0: sort-based coders (default), 1: histogram-pruned coder where it applies.
+// 0: by tile density (default), 1: sort-based coders only, 2: histogram-pruned coder wherever it applies.
 static int g_patch_coder_mode = 0;
+
+// Flags of the kernel chains (see PatchArgs): two words per call, taken in turn from a small ring.
+constexpr int kChainSlots = 256;
+static __device__ unsigned int g_chain_flags[2 * kChainSlots];
+static std::atomic<uint32_t> g_chain_calls{0};
+
+static cudaError_t chain_flags(uint32_t* call_id, unsigned int** first, unsigned int** second) {
+  static unsigned int* base[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!base[dev]) {
+    void* ptr = nullptr;
+    if ((e = cudaGetSymbolAddress(&ptr, g_chain_flags)) != cudaSuccess) return e;
+    base[dev] = static_cast<unsigned int*>(ptr);
+  }
+  uint32_t id = ++g_chain_calls;
+  if (id == 0) id = ++g_chain_calls;  // 0 is what the flags hold before any call
+  *call_id = id;
+  *first = base[dev] + 2 * (id % kChainSlots);
+  *second = *first + 1;
+  return cudaSuccess;
+}
 int patch_coder_mode() { return g_patch_coder_mode; }
 void set_patch_coder_mode(int mode) { g_patch_coder_mode = mode; }
 
@@ -752,6 +832,13 @@ static cudaError_t launch_patches_hist(PatchArgs& a, cudaStream_t stream) {
   return launch_patches(binarize_patches_hist_kernel<BPL, 0>, a, fixed, kWarpsPerCta * 32, kWarpsPerCta, stream);
 }
 
+// Buckets by patch length: enough of them that the few that survive hold well under 256 values.
+static cudaError_t launch_hist_for(PatchArgs& a, cudaStream_t stream) {
+  if (a.n < 1024) return launch_patches_hist<2>(a, stream);
+  if (a.n < 4096) return launch_patches_hist<4>(a, stream);
+  return launch_patches_hist<8>(a, stream);
+}
+
 // The group kernel that codes patches of n > 256 values (the sort-based coder for these lengths, and the one
 // that takes the tiles the other coders mark).
 static cudaError_t launch_group_for(PatchArgs& a, cudaStream_t stream, bool shape_only) {
@@ -786,29 +873,64 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   a.scratch_words = 0;
   a.defer_dense = 0; a.marked_only = 0; a.tile_shape = -1;
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
+  a.dense_num = 1; a.dense_den = 0;  // no tile counts as dense unless a chain below says so
+  a.call_id = 0; a.flag_in = nullptr; a.flag_out = nullptr;
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
-  if (patch_coder_mode() == 1 && a.n <= 8192) {
-    // Histogram-pruned coder on the tile shape of the group kernel, which then takes the tiles left to it.
-    cudaError_t e = launch_group_for(a, stream, /*shape_only=*/true);
-    if (e != cudaSuccess) return e;
-    if ((size_t)a.d.C * ((a.in_h * a.pitch) | 1) <= 65535) {  // its 16-bit offsets reach the whole (odd-pitched) tile
-      e = a.n < 1024 ? launch_patches_hist<2>(a, stream) : launch_patches_hist<4>(a, stream);
+  const int mode = patch_coder_mode();
+  cudaError_t e;
+  if (mode == 1 || a.n > 8192) {
+    // Sort-based coders only.  The patch lengths of the common 3x3 layers (576 values per warp) have variants
+    // without bounds tests whose group size suits rows that are at least half zeros.
+    if (a.n <= 576) {
+      // first the one-warp kernel on the tiles it suits, then four warps per patch on the tiles it marked as dense
+      // (expected non-zeros per patch = density of the staged region * n > 256)
+      a.defer_dense = 1; a.dense_num = 256; a.dense_den = a.n;
+      e = a.n == 576 ? launch_patches_warp<18, true>(a, stream) : launch_patches_warp<18, false>(a, stream);
       if (e != cudaSuccess) return e;
-      a.marked_only = 1;
+      a.defer_dense = 0; a.marked_only = 1;  // a.tile_shape now holds the first kernel's tile
+      return launch_group_for(a, stream, false);
     }
     return launch_group_for(a, stream, false);
   }
-  // The sort-based coders.  The patch lengths of the common 3x3 layers (576 values per warp) have variants
-  // without bounds tests whose group size suits rows that are at least half zeros.  Any other length gets enough
-  // warps for at most 16 values per thread, so that rows with up to half their values non-zero sort with 8 keys
-  // per thread.
+  unsigned int *flag1 = nullptr, *flag2 = nullptr;
+  if ((e = chain_flags(&a.call_id, &flag1, &flag2)) != cudaSuccess) return e;
+  // The histogram-pruned coder runs on the tile shape of the group kernel, which ends every chain by taking the
+  // tiles nobody else settled.  Its 16-bit offsets must reach the whole (odd-pitched) tile.
+  if ((e = launch_group_for(a, stream, /*shape_only=*/true)) != cudaSuccess) return e;
+  const bool hist_fits = (size_t)a.d.C * ((a.in_h * a.pitch) | 1) <= 65535;
+  if (mode == 2) {  // everything through the histogram coder
+    if (hist_fits) {
+      a.flag_out = flag2;
+      e = launch_hist_for(a, stream);
+      if (e != cudaSuccess) return e;
+      a.marked_only = 1; a.flag_in = flag2; a.flag_out = nullptr;
+    }
+    return launch_group_for(a, stream, false);
+  }
+  // By density: the sort-based coder of this length takes the sparse tiles and marks the dense ones; the
+  // histogram coder, whose cost does not grow with the number of non-zero values, takes those; the group kernel
+  // takes what that one leaves.  Tiles count as dense above 256 / n (patches of up to 576 values) or 45 %
+  // non-zero values: about the density from which the sorting kernels need more than 8 keys per thread.
+  if (!hist_fits) {
+    a.tile_shape = -1;
+    return launch_group_for(a, stream, false);
+  }
+  a.defer_dense = 1; a.flag_out = flag1;
   if (a.n <= 576) {
-    // first the one-warp kernel on the tiles it suits, then four warps per patch on the tiles it marked as dense
-    a.defer_dense = 1;
-    cudaError_t e = a.n == 576 ? launch_patches_warp<18, true>(a, stream) : launch_patches_warp<18, false>(a, stream);
+    a.dense_num = 256; a.dense_den = a.n;  // expected non-zeros per patch above the 256 one warp sorts with 8 keys per lane
+    a.tile_shape = -1;  // the one-warp kernel picks its own tile; the two kernels after it take it over
+    e = a.n == 576 ? launch_patches_warp<18, true>(a, stream) : launch_patches_warp<18, false>(a, stream);
+  } else {
+    a.dense_num = 45; a.dense_den = 100;
+    e = launch_group_for(a, stream, false);
+  }
+  if (e != cudaSuccess) return e;
+  a.defer_dense = 0; a.marked_only = 1; a.flag_in = flag1; a.flag_out = nullptr;
+  if ((size_t)a.d.C * ((a.in_h * a.pitch) | 1) <= 65535) {  // (the first kernel may have taken another tile)
+    a.flag_out = flag2;
+    e = launch_hist_for(a, stream);
     if (e != cudaSuccess) return e;
-    a.defer_dense = 0; a.marked_only = 1;  // a.tile_shape now holds the first kernel's tile
-    return launch_patches_group<4, 8, 5, false, true>(a, stream);
+    a.flag_in = flag2; a.flag_out = nullptr;
   }
   return launch_group_for(a, stream, false);
 }

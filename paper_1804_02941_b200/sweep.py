@@ -144,6 +144,7 @@ def main():
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--batch5", type=int, default=256)
     ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"])
+    ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist"])
     ap.add_argument("--stages", default="", help="comma-separated stage names of the convolution layers to run (default all)")
     ap.add_argument("--layers", default="", help="comma-separated layer names to run (default all)")
     args = ap.parse_args()
@@ -151,6 +152,7 @@ def main():
     STAGES = set(args.stages.split(",")) if args.stages else None
     LAYERS = set(args.layers.split(",")) if args.layers else None
     dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
+    dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST}[args.patch_coder])
     want = set(args.configs.split(","))
     hbm, mhz, src = peaks()
     tops_peak = POPC_PER_CLK * WORDS_PER_POPC * SM_COUNT * mhz * 1e6 * 64 / 1e12

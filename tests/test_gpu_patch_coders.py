@@ -1,5 +1,5 @@
-"""The two patch coders (full sort, histogram-pruned search) must give the same codes bit for bit, and the
-histogram coder must match the CPU checker on its own."""
+"""The patch coders (full sort, histogram-pruned search, the default choice between them by tile density) must give
+the same codes bit for bit, and the histogram coder must match the CPU checker on its own."""
 import numpy as np
 import pytest
 import torch
@@ -17,7 +17,7 @@ def dab():
     d.lib()
     oracle.set_threads(8)
     yield d
-    d.dab_set_patch_coder(d.PATCHES_SORT)
+    d.dab_set_patch_coder(d.PATCHES_AUTO)
 
 
 def _code(dab, x, C, kh, kw, stride, pad, coder):
@@ -33,7 +33,7 @@ def _code(dab, x, C, kh, kw, stride, pad, coder):
     pf = torch.zeros(P, dtype=torch.int32, device=dev)
     dab.dab_binarize_patches(desc, x, pK, pg, pd, pm, pf)
     torch.cuda.synchronize()
-    dab.dab_set_patch_coder(dab.PATCHES_SORT)
+    dab.dab_set_patch_coder(dab.PATCHES_AUTO)
     return pK, pg, pd, pm, pf
 
 
@@ -73,8 +73,9 @@ def test_histogram_coder_equals_sort_coder_and_checker(dab, ci):
     xd = to_dev(x)
     a = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_SORT)
     b = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_HIST)
-    for s, h in zip(a, b):
-        assert torch.equal(s, h)
+    c = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_AUTO)
+    for s, h, au in zip(a, b, c):
+        assert torch.equal(s, h) and torch.equal(s, au)
     n = C * kh * kw
     rows = oracle.im2col(x, kh, kw, stride, pad)
     sel = np.unique(np.concatenate([[0, len(rows) - 1], (dab_synth.uniform01(96, ci, 0, 64) * len(rows)).astype(np.int64)]))
@@ -93,5 +94,24 @@ def test_nonfinite_tiles_fall_back(dab):
     xd = to_dev(x)
     a = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
     b = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_HIST)
+    c = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
     assert torch.equal(a[0], b[0]) and torch.equal(a[3], b[3]) and torch.equal(a[4], b[4])
+    assert torch.equal(a[0], c[0]) and torch.equal(a[3], c[3]) and torch.equal(a[4], c[4])
     assert int((b[4] == 2).sum()) == 9 + 4
+
+
+def test_mixed_density_batches_split_between_the_coders(dab):
+    # images of very different density in one call: every tile goes to one coder or the other
+    x = np.concatenate([dab_synth.relu_activations((1, 128, 14, 14), z, stream=995 + i) for i, z in
+                        enumerate((0.9, 0.6, 0.5, 0.3, 0.0))]).astype(np.float32)
+    x[4] = dab_synth.normal((128, 14, 14), 1.0, stream=999)
+    xd = to_dev(x)
+    a = _code(dab, xd, 128, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
+    c = _code(dab, xd, 128, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
+    for s, au in zip(a, c):
+        assert torch.equal(s, au)
+    x64 = np.ascontiguousarray(x[:, :64])
+    a = _code(dab, to_dev(x64), 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
+    c = _code(dab, to_dev(x64), 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
+    for s, au in zip(a, c):
+        assert torch.equal(s, au)
