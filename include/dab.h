@@ -293,7 +293,7 @@ dab_contraction dab_get_contraction(void);
  *   DAB_PATCHES_HIST   patches of 257..8192 values go through a histogram of their values that bounds the
  *                      objective per bucket (it is convex in the split size and the prefix sum) and leaves only
  *                      the few buckets that can hold the maximum to the exact search; tiles it cannot settle (a
- *                      hull of more than 256 values, non-finite inputs) fall to the sorting kernel.  Its cost does
+ *                      hull of more than 256 (patches of fewer than 1024 values) or 1024 values, non-finite inputs) fall to the sorting kernel.  Its cost does
  *                      not grow with the number of non-zero values: 2.5x to 6.5x faster than sorting on inputs
  *                      without zeros, about 10 % slower on inputs that are 60 % zeros;
  *   DAB_PATCHES_AUTO   (default) per tile of the input: the sorting kernels take the tiles with few non-zero

@@ -1,5 +1,6 @@
-// dab_binarize: the row coder of rowcode.cuh applied to the rows of a matrix (one warp per row for up to 1024
-// values, a group of 2..16 warps beyond).
+// dab_binarize: the rows of a matrix through the sorting coder of rowcode.cuh (one warp per row for up to 256
+// values, a group of 4..32 warps beyond) or, for large dense matrices, the histogram-pruned search of histcode.cuh.
+#include "histcode.cuh"
 #include "rowcode.cuh"
 
 namespace dab {
@@ -11,7 +12,9 @@ template <int R, bool kFull>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
     const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
     float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
-    uint32_t* __restrict__ flags_out) {
+    uint32_t* __restrict__ flags_out, const unsigned int* marked_flag, uint32_t call_id) {
+  // marked_flag: code only the rows an earlier kernel of the call marked (K = kRowMark), and leave at once if it marked none
+  if (marked_flag && *reinterpret_cast<const volatile unsigned int*>(marked_flag) != call_id) return;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
   uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + rcp_table_slots(n));
@@ -21,6 +24,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
   __syncthreads();
 
   for (int64_t row = (int64_t)blockIdx.x * kWarpsPerCta + warp; row < rows; row += (int64_t)gridDim.x * kWarpsPerCta) {
+    if (marked_flag && K_out[row] != kRowMark) continue;
     const float* v = values + row * ld_values;
     auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
     uint32_t kreg[R];
@@ -44,7 +48,8 @@ template <int W, int WARPS, int R, bool kFull, bool kTable>
 __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
     const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
     float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
-    uint32_t* __restrict__ flags_out, int scratch_words) {
+    uint32_t* __restrict__ flags_out, int scratch_words, const unsigned int* marked_flag, uint32_t call_id) {
+  if (marked_flag && *reinterpret_cast<const volatile unsigned int*>(marked_flag) != call_id) return;
   constexpr int G = WARPS / W;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
@@ -62,6 +67,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
   }
 
   for (int64_t row = (int64_t)blockIdx.x * G + group; row < rows; row += (int64_t)gridDim.x * G) {
+    if (marked_flag && K_out[row] != kRowMark) continue;  // the same for every thread of the group
     const float* v = values + row * ld_values;
     auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
     uint32_t kreg[R];
@@ -81,7 +87,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
 template <int R, bool kFull>
 static cudaError_t launch_rows_warp(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                     float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                                    cudaStream_t stream) {
+                                    cudaStream_t stream, const unsigned int* marked_flag, uint32_t call_id) {
   auto kern = binarize_rows_warp_kernel<R, kFull>;
   size_t smem = sizeof(double) * rcp_table_slots(n) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -89,14 +95,14 @@ static cudaError_t launch_rows_warp(const float* values, int64_t rows, int32_t n
   int64_t blocks = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
   if (blocks > 148 * 16) blocks = 148 * 16;
   kern<<<(unsigned)blocks, kWarpsPerCta * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask,
-                                                              ld_mask, flags);
+                                                              ld_mask, flags, marked_flag, call_id);
   return cudaGetLastError();
 }
 
 template <int W, int WARPS, int R, bool kFull, bool kTable>
 static cudaError_t launch_rows_group(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                      float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                                     cudaStream_t stream) {
+                                     cudaStream_t stream, const unsigned int* marked_flag, uint32_t call_id) {
   constexpr int G = WARPS / W;
   auto kern = binarize_rows_group_kernel<W, WARPS, R, kFull, kTable>;
   int sw = scratch_words_for(n, W);
@@ -106,14 +112,119 @@ static cudaError_t launch_rows_group(const float* values, int64_t rows, int32_t 
   int64_t blocks = (rows + G - 1) / G;
   if (blocks > 148 * 16) blocks = 148 * 16;
   kern<<<(unsigned)blocks, WARPS * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask,
-                                                       flags, sw);
+                                                       flags, sw, marked_flag, call_id);
   return cudaGetLastError();
 }
 
-cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
-                            float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                            cudaStream_t stream) {
-#define DAB_ARGS values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream
+// ---------------------------------------------------------------------------------------------------------
+// Rows of a matrix through the histogram-pruned search of histcode.cuh, one warp per row.  Four passes over the
+// row (read through the caches): range of the non-zero values, histogram, gather of the hull, mask.  Rows it
+// does not settle (a NaN or an infinity, a hull of more than 256 or 1024 values, too few non-zero values when
+// min_density_pct is set) are marked with K = kRowMark for the sorting kernel that follows it on the stream.
+// ---------------------------------------------------------------------------------------------------------
+template <int BPL>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kernel(
+    const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
+    float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
+    uint32_t* __restrict__ flags_out, int min_density_pct, unsigned int* flag_out, uint32_t call_id) {
+  constexpr int B = 32 * BPL;
+  constexpr int LOG2B = BPL == 1 ? 5 : BPL == 2 ? 6 : BPL == 4 ? 7 : 8;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* rcp = reinterpret_cast<double*>(smem_raw);
+  int2* hist_all = reinterpret_cast<int2*>(rcp + rcp_table_slots(n));
+  uint32_t* scratch_all = reinterpret_cast<uint32_t*>(hist_all + kWarpsPerCta * B);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int2* hist = hist_all + warp * B;
+  uint32_t* scratch = scratch_all + warp * hist_cap(BPL);
+  fill_reciprocals(rcp, n, threadIdx.x, blockDim.x);
+  __syncthreads();
+  const int qbits = quant_bits(n, LOG2B);
+  const int rounds = (n + 31) >> 5;
+
+  for (int64_t row = (int64_t)blockIdx.x * kWarpsPerCta + warp; row < rows; row += (int64_t)gridDim.x * kWarpsPerCta) {
+    const float* v = values + row * ld_values;
+    auto element = [v, n, lane](int k) {  // element of round k for this lane (+0.0 folds -0.0), 0.0 beyond the row
+      const int i = k * 32 + lane;
+      return i < n ? __fadd_rn(__ldg(v + i), 0.0f) : 0.0f;
+    };
+    // pass 0: range and number of the non-zero values
+    uint32_t kmin = kPadKey, kmax = 0u;
+    int nz = 0;
+#pragma unroll 4
+    for (int k = 0; k < rounds; ++k) {
+      const float x = element(k);
+      if (x != 0.0f) {  // NaN compares unequal: counted, and seen as non-finite below
+        const uint32_t key = order_key(x);
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
+        ++nz;
+      }
+    }
+    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+    nz = __reduce_add_sync(0xFFFFFFFFu, nz);
+    const bool any_nonzero = kmin <= kmax;
+    bool retry = (any_nonzero && key_range_nonfinite(kmin, kmax)) || (int64_t)nz * 100 < (int64_t)min_density_pct * n;
+    RowResult res;
+    if (!retry) {
+      const Quant qz = make_quant(any_nonzero ? key_value(kmin) : 0.0f, any_nonzero ? key_value(kmax) : 0.0f, qbits, LOG2B);
+      auto sweep = [&](auto f) {
+#pragma unroll 4
+        for (int k = 0; k < rounds; ++k) f(element(k), k * 32 + lane < n);
+      };
+      retry = !hist_search<BPL>(sweep, n, qz, hist, scratch, rcp, lane, res);
+    }
+    if (retry) {
+      if (lane == 0) {
+        K_out[row] = kRowMark;
+        *flag_out = call_id;
+      }
+      continue;
+    }
+    if (lane == 0) {
+      K_out[row] = res.K;
+      alpha_out[row] = res.alpha;
+      beta_out[row] = res.beta;
+      if (flags_out) flags_out[row] = res.flags;
+    }
+    const bool flip = res.mode == 1, none = res.mode == 2;
+    const float tv = key_value(res.tkey);
+    uint32_t* mrow = mask_out + row * (int64_t)ld_mask;
+    uint32_t mine = 0;
+#pragma unroll 4
+    for (int k = 0; k < rounds; ++k) {
+      const float x = element(k);
+      const bool bit = !none && (k * 32 + lane < n) && ((x >= tv) != flip);
+      const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
+      if ((k & 31) == lane) mine = word;
+      if ((k & 31) == 31 || k == rounds - 1) {
+        const int w = (k & ~31) + lane;
+        if (w <= k) mrow[w] = mine;
+      }
+    }
+    for (int w = rounds + lane; w < ld_mask; w += 32) mrow[w] = 0u;
+  }
+}
+
+template <int BPL>
+static cudaError_t launch_rows_hist(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
+                                    float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
+                                    cudaStream_t stream, int min_density_pct, unsigned int* flag_out, uint32_t call_id) {
+  auto kern = binarize_rows_hist_kernel<BPL>;
+  size_t smem = sizeof(double) * rcp_table_slots(n) + (sizeof(int2) * 32 * BPL + sizeof(uint32_t) * hist_cap(BPL)) * kWarpsPerCta;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int64_t blocks = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  kern<<<(unsigned)blocks, kWarpsPerCta * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask,
+                                                              ld_mask, flags, min_density_pct, flag_out, call_id);
+  return cudaGetLastError();
+}
+
+static cudaError_t launch_rows_sort(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
+                                    float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
+                                    cudaStream_t stream, const unsigned int* marked_flag, uint32_t call_id) {
+#define DAB_ARGS values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, marked_flag, call_id
   // A matrix may have few rows (a layer's filters), so a row gets enough warps for at most 8 keys per thread
   // even when none of its values is zero: short critical path per row, and the 8-key network is the most
   // efficient one per element.
@@ -124,6 +235,29 @@ cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_
   if (n <= 8192) return launch_rows_group<32, 32, 8, false, true>(DAB_ARGS);
   return launch_rows_group<32, 32, 16, false, false>(DAB_ARGS);
 #undef DAB_ARGS
+}
+
+// Rows at which a matrix is large enough for one warp per row to fill the device: below it the sorting kernels,
+// which put up to 32 warps on a row, finish sooner.
+constexpr int64_t kHistMinRows = 2048;
+
+cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
+                            float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
+                            cudaStream_t stream) {
+  const int mode = patch_coder_mode();  // the setting covers the rows of matrices as well
+  if (mode == 1 || n <= 256 || n > 8192 || (mode == 0 && rows < kHistMinRows))
+    return launch_rows_sort(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, nullptr, 0);
+  // The histogram-pruned search first; the sorting kernel then takes the rows it marked.
+  uint32_t call_id = 0;
+  unsigned int *flag1 = nullptr, *flag2 = nullptr;
+  cudaError_t e = chain_flags(&call_id, &flag1, &flag2);
+  if (e != cudaSuccess) return e;
+  const int min_density = 0;  // rows of any density: on matrices this large the search beats the sort on sparse rows too
+  if (n < 1024) e = launch_rows_hist<2>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density, flag1, call_id);
+  else if (n < 4096) e = launch_rows_hist<4>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density, flag1, call_id);
+  else e = launch_rows_hist<8>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density, flag1, call_id);
+  if (e != cudaSuccess) return e;
+  return launch_rows_sort(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, flag1, call_id);
 }
 
 }  // namespace dab

@@ -94,6 +94,9 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
 // Patch coder selection: 0 by tile density (default), 1 sort-based only, 2 histogram-pruned wherever it applies.
 int patch_coder_mode();
 void set_patch_coder_mode(int mode);
+// Two flag words for a chain of kernels of one call (see PatchArgs in patches.cu) and the call's id.
+cudaError_t chain_flags(uint32_t* call_id, unsigned int** first, unsigned int** second);
+constexpr int32_t kRowMark = -1;  // K of a row or of a tile's first patch that the next kernel of a chain has to code
 cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K, float* alpha,
                              float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags, cudaStream_t stream);
 cudaError_t launch_sign_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,

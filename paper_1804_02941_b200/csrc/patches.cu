@@ -2,6 +2,7 @@
 // (one warp per patch for up to 1024 values, a group of 2..16 warps beyond).
 #include <atomic>
 
+#include "histcode.cuh"
 #include "rowcode.cuh"
 
 namespace dab {
@@ -246,48 +247,15 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Histogram-pruned patch coder.  One warp per patch, three passes over the patch in the staged tile:
-//   1. every non-zero value is quantised (q = floor(v * qscale), a fixed scale per tile) and counted into one of
-//      B = 32*BPL buckets (bucket = high bits of q): per bucket the count and the sum of the low bits of q, by
-//      shared-memory atomics;
-//   2. a scan over the buckets gives, at every bucket edge, the split size s exactly and the prefix sum P to
-//      within the quantisation error, hence the objective there to within a known eps; inside a bucket the
-//      objective is bounded by its values at the corners of the parallelogram that the bucket's value range
-//      allows (the objective is jointly convex in (s, P)).  Buckets whose bound cannot reach the best edge value
-//      are discarded; the hull of the others (usually two or three buckets) is gathered, with exact fp64 sums of
-//      everything below and above it, sorted and searched by the exact evaluator of rowcode.cuh;
-//   3. the mask is a threshold compare, as in the other coders.
-// Discarding is conservative (every rounding is covered by eps), so the result is the same split the full
-// search finds.  Patches whose hull exceeds 256 values, and tiles holding a NaN or an infinity, are left to the
+// Histogram-pruned patch coder: the search of histcode.cuh, one warp per patch, on the staged tile (one
+// quantisation per tile, from the range of its non-zero values), then the mask as a threshold compare as in
+// the other coders.  Patches the search does not settle, and tiles holding a NaN or an infinity, are left to the
 // group kernel through the dense-tile mark.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kHistCap = 256;  // keys the exact search takes at most
-
 struct HistTile {          // per tile, in shared memory
   uint32_t kmin, kmax;     // smallest and largest key among the non-zero staged values
   int retry;               // some patch of the tile could not be coded here
 };
-
-__device__ __forceinline__ float objective_f32(float s, float P, float T, float n) {
-  // P^2/s + (T-P)^2/(n-s) with the limits 0 at s = 0 (P = 0 there) and s = n
-  const float Q = T - P;
-  const float a = s > 0.0f ? __fdividef(P * P, s) : 0.0f;
-  const float b = n - s > 0.0f ? __fdividef(Q * Q, n - s) : 0.0f;
-  return a + b;
-}
-
-template <int E>
-__device__ __noinline__ RowResult hist_sort_select(const uint32_t* scratch, int m, int z, int n, int lane,
-                                                   const double* rcp, const SplitBase base) {
-  uint32_t r[E];
-#pragma unroll
-  for (int j = 0; j < E; ++j) {
-    const int idx = j * 32 + lane;
-    r[j] = idx < m ? order_key(__uint_as_float(scratch[idx])) : kPadKey;   // the gather stored raw bits
-  }
-  group_sort<1, E>(r, lane, nullptr, 0);
-  return group_select<1, E, true, true>(r, m, z, n, lane, nullptr, 0, rcp, base);
-}
 
 #ifndef DAB_HIST_MINBLOCKS
 #define DAB_HIST_MINBLOCKS 3  // CTAs per SM the histogram coder is compiled for (register budget)
@@ -304,7 +272,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
   double* rcp = reinterpret_cast<double*>(smem_raw);
   int2* hist_all = reinterpret_cast<int2*>(rcp + rcp_table_slots(a.n));          // [warp][B] (count, sum of offsets)
   uint32_t* scratch_all = reinterpret_cast<uint32_t*>(hist_all + kWarpsPerCta * B);
-  float* tile = reinterpret_cast<float*>(scratch_all + kWarpsPerCta * kHistCap);
+  float* tile = reinterpret_cast<float*>(scratch_all + kWarpsPerCta * hist_cap(BPL));
   const int ch_words = (a.in_h * a.pitch) | 1;  // odd: the 32 channels a warp reads at once fall into 32 banks
   uint16_t* off = reinterpret_cast<uint16_t*>(tile + (size_t)a.d.C * ch_words);
   uint16_t* win = off + ((a.n + 1) & ~1);       // offsets of the kernel window inside one channel
@@ -313,7 +281,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
   if (a.marked_only && !has_marked_tile(a)) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int2* hist = hist_all + warp * B;
-  uint32_t* scratch = scratch_all + warp * kHistCap;
+  uint32_t* scratch = scratch_all + warp * hist_cap(BPL);
   const int khw = a.d.kh * a.d.kw;
   fill_reciprocals(rcp, a.n, threadIdx.x, THREADS);
   fill_offsets(a, off, ch_words, threadIdx.x, THREADS);
@@ -322,12 +290,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
   int wofs[KMAX];
 #pragma unroll
   for (int rs = 0; rs < KMAX; ++rs) wofs[rs] = KHW ? win[rs] : 0;
-  // bits of q: 24 (fp32 holds them), fewer if the sum of n in-bucket offsets (qbits - log2 B bits each) could leave 32 bits
-  int qbits = 24;
-  while (((int64_t)a.n << (qbits - LOG2B)) >= 0x7FFFFFFFll) --qbits;
+  const int qbits = quant_bits(a.n, LOG2B);
   const int rounds = (a.n + 31) >> 5;
-  const float nf = (float)a.n;
-  const unsigned lt = (1u << lane) - 1u;
 
   const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
@@ -374,25 +338,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
       }
       continue;
     }
-    // Quantisation of the tile: q = floor(v * qscale); bucket = (q >> shift) + boff; B0 = first bucket of positives.
     const float lo = any_nonzero ? key_value(tkmin) : 0.0f, hi = any_nonzero ? key_value(tkmax) : 0.0f;
-    float qscale;
-    int boff, B0;
-    const int shift = qbits - LOG2B;
-    if (lo >= 0.0f) {         // no negative value: q in [0, 2^qbits)
-      qscale = __fdividef((float)(1 << qbits) * 0.99999f, fmaxf(hi, 1e-37f));
-      boff = 0; B0 = 0;
-    } else if (hi <= 0.0f) {  // no positive value: q in [-2^qbits, 0)
-      qscale = __fdividef((float)(1 << qbits) * 0.99999f, -lo);
-      boff = B; B0 = B;
-    } else {                  // both signs: q in [-2^(qbits-1), 2^(qbits-1))
-      qscale = __fdividef((float)(1 << (qbits - 1)) * 0.99999f, fmaxf(-lo, hi));
-      boff = B / 2; B0 = B / 2;
-    }
-    const float u = __fdividef(1.0f, qscale);              // value of one unit of q
-    const int qmask = (1 << shift) - 1;
-    const float bw = (float)(1 << shift);                  // bucket width in units of q
-    const float A = fmaxf(fabsf(lo), fabsf(hi)), R = hi - lo;
+    const Quant qz = make_quant(lo, hi, qbits, LOG2B);  // one quantisation for the tile
 
     for (int p = warp; p < t.th * t.tw; p += kWarpsPerCta) {
       const int lh = p / t.tw, lw = p % t.tw;
@@ -400,191 +347,21 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
       const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
       uint32_t* mrow = a.pmask + pi * (int64_t)a.ldp;
 
-      // ---- pass 1: histogram (the order of the elements does not matter: lane = channel, loop over the window) ----
+      // the two sweeps of the search take the elements in any order: lane = channel, loop over the kernel window
+      auto sweep = [&](auto f) {
+        for (int c0 = 0; c0 < a.d.C; c0 += 32) {
+          const bool cin = c0 + lane < a.d.C;
+          const float* src = origin + (cin ? c0 + lane : 0) * ch_words;
+          if (KHW) {
 #pragma unroll
-      for (int j = 0; j < BPL; ++j) hist[lane * BPL + j] = make_int2(0, 0);
-      __syncwarp();
-      for (int c0 = 0; c0 < a.d.C; c0 += 32) {
-        const bool cin = c0 + lane < a.d.C;
-        const float* src = origin + (cin ? c0 + lane : 0) * ch_words;
-        auto tally = [&](float v) {
-          const int q = __float2int_rd(v * qscale);
-          const int b = min(max((q >> shift) + boff, 0), B - 1);
-          if (cin && v != 0.0f) {
-            atomicAdd(&hist[b].x, 1);
-            atomicAdd(&hist[b].y, q & qmask);
-          }
-        };
-        if (KHW) {
-#pragma unroll
-          for (int rs = 0; rs < KMAX; ++rs) tally(src[wofs[rs]]);
-        } else {
-          for (int rs = 0; rs < khw; ++rs) tally(src[win[rs]]);
-        }
-      }
-      __syncwarp();
-      // ---- scan over the buckets: lane owns buckets lane*BPL .. lane*BPL+BPL-1 ----
-      int c[BPL];
-      double Q[BPL];   // sum of q over the bucket: count * first q of the bucket + sum of the offsets (exact)
-      int csum = 0;
-      double qsum = 0.0;
-#pragma unroll
-      for (int j = 0; j < BPL; ++j) {
-        const int2 hq = hist[lane * BPL + j];
-        c[j] = hq.x;
-        Q[j] = (double)hq.x * (double)((lane * BPL + j - boff) * (1 << shift)) + (double)(unsigned)hq.y;
-        csum += hq.x; qsum += Q[j];
-      }
-      int cincl = csum;
-      double qincl = qsum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int co = __shfl_up_sync(0xFFFFFFFFu, cincl, o);
-        const double qo = __shfl_up_sync(0xFFFFFFFFu, qincl, o);
-        if (lane >= o) { cincl += co; qincl += qo; }
-      }
-      const int m = __shfl_sync(0xFFFFFFFFu, cincl, 31);
-      const double QT = __shfl_sync(0xFFFFFFFFu, qincl, 31);
-      const int z = a.n - m;
-      RowResult res;
-      bool retry = false;
-      if (m == 0) {
-        res = trivial_row(false, 0.0f);  // nothing but zeros
-      } else {
-        // nominal prefix sums in units of u: every value lies in [(q - 1) u, (q + 2) u], centre (q + 0.5) u
-        const float Tn = ((float)QT + 0.5f * (float)m) * u;
-        const float eps_fixed = 3.0f * (R + A) * (float)m * u;          // effect of the quantisation on any objective value
-        int cbefore = cincl - csum;
-        double qbefore = qincl - qsum;
-        float best_edge = -1.0f;
-        float bound[BPL];
-        int negc_local = 0;
-#pragma unroll
-        for (int j = 0; j < BPL; ++j) {
-          const int b = lane * BPL + j;
-          const float s0 = (float)(cbefore + (b >= B0 ? z : 0));
-          const float P0 = ((float)qbefore + 0.5f * (float)cbefore) * u;
-          const int cafter = cbefore + c[j];
-          const double qafter = qbefore + Q[j];
-          const float s1 = s0 + (float)c[j];
-          const float P1 = ((float)qafter + 0.5f * (float)cafter) * u;
-          float d0 = -1.0f, d1 = -1.0f, dk = -1.0f;
-          if (s0 > 0.0f && s0 < nf) d0 = objective_f32(s0, P0, Tn, nf);
-          if (s1 > 0.0f && s1 < nf) d1 = objective_f32(s1, P1, Tn, nf);
-          best_edge = fmaxf(best_edge, fmaxf(d0, d1));
-          if (c[j] >= 2) {
-            // value range of the bucket, and the two inner corners of the region (s, P) can visit inside it
-            const float qlo = (float)(b - boff) * bw;
-            const float va = (qlo - 1.0f) * u, vb = (qlo + bw + 2.0f) * u;
-            const float cf = (float)c[j], sig = P1 - P0;
-            float jl = __fdividef(cf * vb - sig, vb - va);
-            jl = fminf(fmaxf(jl, 0.0f), cf);
-            const float ju = cf - jl;
-            dk = fmaxf(objective_f32(s0 + jl, P0 + jl * va, Tn, nf), objective_f32(s0 + ju, P0 + ju * vb, Tn, nf));
-            // the corners move with the uncertainty of the bucket's sum: 1.5 c u in P, that over (vb - va) in s
-            dk += (A * A + 2.0f * R * A) * __fdividef(1.5f * cf * u, vb - va) + 2.0f * R * 1.5f * cf * u;
-          }
-          bound[j] = c[j] > 0 ? fmaxf(fmaxf(d0, d1), dk) : -2.0f;
-          if (b < B0) negc_local += c[j];
-          cbefore = cafter; qbefore = qafter;
-        }
-        const int negc = __reduce_add_sync(0xFFFFFFFFu, negc_local);
-        // the two splits around the run of zeros (their sums are those of the negatives)
-        const double qneg = __shfl_sync(0xFFFFFFFFu, qincl, max(B0 / BPL - 1, 0));   // inclusive sum up to bucket B0-1
-        const float Pneg = B0 > 0 ? ((float)qneg + 0.5f * (float)negc) * u : 0.0f;
-        float dz0 = -1.0f, dz1 = -1.0f;
-        if (z > 0) {
-          if (negc > 0) dz0 = objective_f32((float)negc, Pneg, Tn, nf);
-          if (negc + z < a.n) dz1 = objective_f32((float)(negc + z), Pneg, Tn, nf);
-        }
-        best_edge = fmaxf(best_edge, fmaxf(dz0, dz1));
-        best_edge = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fmaxf(best_edge, 0.0f))));
-        // a bucket (or the zero run) survives if its bound, raised by every rounding, reaches the best edge lowered by them
-        const float slack = 2.0f * eps_fixed + 2e-4f * best_edge;
-        const float need = best_edge - slack;
-        int seg_lo = 1 << 20, seg_hi = -1;
-#pragma unroll
-        for (int j = 0; j < BPL; ++j) {
-          const int b = lane * BPL + j;
-          if (c[j] > 0 && bound[j] + slack >= need) {
-            const int seg = b + (b >= B0 ? 1 : 0);
-            seg_lo = min(seg_lo, seg);
-            seg_hi = max(seg_hi, seg);
-          }
-        }
-        if (z > 0 && fmaxf(dz0, dz1) + slack >= need) { seg_lo = min(seg_lo, B0); seg_hi = max(seg_hi, B0); }
-        seg_lo = __reduce_min_sync(0xFFFFFFFFu, seg_lo);
-        seg_hi = __reduce_max_sync(0xFFFFFFFFu, seg_hi);
-        // hull in bucket and q terms
-        const int b_lo = seg_lo > B0 ? seg_lo - 1 : seg_lo;          // first bucket of the hull (seg_lo == B0: bucket B0)
-        const int b_hi = seg_hi >= B0 ? seg_hi - 1 : seg_hi;         // last bucket of the hull (seg_hi == B0: bucket B0-1)
-        const int z_in = (z > 0 && seg_lo <= B0 && B0 <= seg_hi) ? z : 0;
-        int msub_local = 0, sbelow_local = 0;
-#pragma unroll
-        for (int j = 0; j < BPL; ++j) {
-          const int b = lane * BPL + j;
-          if (b >= b_lo && b <= b_hi) msub_local += c[j];
-          if (b < b_lo) sbelow_local += c[j];
-        }
-        const int m_sub = __reduce_add_sync(0xFFFFFFFFu, msub_local);
-        int s_below = __reduce_add_sync(0xFFFFFFFFu, sbelow_local);
-        if (seg_lo > B0) s_below += z;                               // the zeros lie below the hull
-        // (a constant row has all its values in one bucket: with more than kHistCap values it is left to the group kernel)
-        if (seg_hi < 0 || m_sub < 1 || m_sub > kHistCap || (z == 0 && m_sub == a.n)) {
-          retry = true;
-        } else {
-          const int qA = (b_lo - boff) * (1 << shift);               // q range of the hull's buckets
-          const int qB = (b_hi + 1 - boff) * (1 << shift) - 1;
-          const bool open_lo = b_lo == 0, open_hi = b_hi == B - 1;   // the end buckets take whatever falls outside the range
-          // ---- pass 2: gather the hull (raw bits), exact sums of what lies below and above it ----
-          double below = 0.0, above = 0.0;
-          int cnt = 0;
-          for (int c0 = 0; c0 < a.d.C; c0 += 32) {
-            const bool cin = c0 + lane < a.d.C;
-            const float* src = origin + (cin ? c0 + lane : 0) * ch_words;
-            auto sift = [&](float v) {
-              const int q = __float2int_rd(v * qscale);
-              const bool nz = cin && v != 0.0f;
-              const bool lowq = nz && q < qA && !open_lo, highq = nz && q > qB && !open_hi;
-              const bool in = nz && !lowq && !highq;
-              const double dv = (double)v;
-              below = __dadd_rn(below, lowq ? dv : 0.0);
-              above = __dadd_rn(above, highq ? dv : 0.0);
-              const unsigned bal = __ballot_sync(0xFFFFFFFFu, in);
-              if (in) scratch[min(cnt + __popc(bal & lt), kHistCap - 1)] = __float_as_uint(v);
-              cnt += __popc(bal);
-            };
-            if (KHW) {
-#pragma unroll
-              for (int rs = 0; rs < KMAX; ++rs) sift(src[wofs[rs]]);
-            } else {
-              for (int rs = 0; rs < khw; ++rs) sift(src[win[rs]]);
-            }
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            below = __dadd_rn(below, __shfl_xor_sync(0xFFFFFFFFu, below, o));
-            above = __dadd_rn(above, __shfl_xor_sync(0xFFFFFFFFu, above, o));
-          }
-          __syncwarp();
-          if (cnt != m_sub) {
-            retry = true;                                            // cannot happen; never trust a mismatch
+            for (int rs = 0; rs < KMAX; ++rs) f(src[wofs[rs]], cin);
           } else {
-            const SplitBase base{s_below, below, above};
-            if (m_sub <= 64) res = hist_sort_select<2>(scratch, m_sub, z_in, a.n, lane, rcp, base);
-            else if (m_sub <= 128) res = hist_sort_select<4>(scratch, m_sub, z_in, a.n, lane, rcp, base);
-            else res = hist_sort_select<8>(scratch, m_sub, z_in, a.n, lane, rcp, base);
-            res.K = __shfl_sync(0xFFFFFFFFu, res.K, 0);
-            res.alpha = __shfl_sync(0xFFFFFFFFu, res.alpha, 0);
-            res.beta = __shfl_sync(0xFFFFFFFFu, res.beta, 0);
-            res.flags = 0u;
-            res.tkey = __shfl_sync(0xFFFFFFFFu, res.tkey, 0);
-            res.mode = __shfl_sync(0xFFFFFFFFu, res.mode, 0);
-            if (res.tkey == kPadKey) retry = true;                   // a split at the hull's outer edge won: not certified
+            for (int rs = 0; rs < khw; ++rs) f(src[win[rs]], cin);
           }
-          __syncwarp();
         }
-      }
+      };
+      RowResult res;
+      const bool retry = !hist_search<BPL>(sweep, a.n, qz, hist, scratch, rcp, lane, res);
       if (retry) {
         if (lane == 0) ht.retry = 1;
         continue;
@@ -722,7 +499,7 @@ constexpr int kChainSlots = 256;
 static __device__ unsigned int g_chain_flags[2 * kChainSlots];
 static std::atomic<uint32_t> g_chain_calls{0};
 
-static cudaError_t chain_flags(uint32_t* call_id, unsigned int** first, unsigned int** second) {
+cudaError_t chain_flags(uint32_t* call_id, unsigned int** first, unsigned int** second) {
   static unsigned int* base[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -825,14 +602,14 @@ template <int BPL>
 static cudaError_t launch_patches_hist(PatchArgs& a, cudaStream_t stream) {
   // beyond the group kernel's tile: one more word per channel (odd channel pitch) and the window offsets
   size_t fixed = sizeof(double) * rcp_table_slots(a.n) + sizeof(int2) * 32 * BPL * kWarpsPerCta +
-                 sizeof(uint32_t) * kHistCap * kWarpsPerCta + sizeof(float) * a.d.C +
+                 sizeof(uint32_t) * hist_cap(BPL) * kWarpsPerCta + sizeof(float) * a.d.C +
                  sizeof(uint16_t) * (size_t)(a.d.kh * a.d.kw + 2);
   if (a.d.kh * a.d.kw == 9)
     return launch_patches(binarize_patches_hist_kernel<BPL, 9>, a, fixed, kWarpsPerCta * 32, kWarpsPerCta, stream);
   return launch_patches(binarize_patches_hist_kernel<BPL, 0>, a, fixed, kWarpsPerCta * 32, kWarpsPerCta, stream);
 }
 
-// Buckets by patch length: enough of them that the few that survive hold well under 256 values.
+// Buckets by patch length: enough of them that the few that survive hold well under the 256 or 1024 values the exact search takes.
 static cudaError_t launch_hist_for(PatchArgs& a, cudaStream_t stream) {
   if (a.n < 1024) return launch_patches_hist<2>(a, stream);
   if (a.n < 4096) return launch_patches_hist<4>(a, stream);

@@ -115,3 +115,59 @@ def test_mixed_density_batches_split_between_the_coders(dab):
     c = _code(dab, to_dev(x64), 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
     for s, au in zip(a, c):
         assert torch.equal(s, au)
+
+
+@pytest.mark.parametrize("n", [257, 300, 575, 576, 577, 1024, 1152, 1600, 2304, 4096, 4608, 8192])
+@pytest.mark.parametrize("kind", ["normal", "relu", "laplace", "ints", "cluster", "negative"])
+def test_rows_of_a_matrix_through_both_coders(dab, n, kind):
+    # dab_binarize: the histogram-pruned search against the sorting kernels and against the checker
+    from parity_util import check_coded
+    rows = 40 if n <= 2304 else 12
+    if kind == "normal":
+        w = dab_synth.normal((rows, n), 0.05, stream=n)
+    elif kind == "relu":
+        w = dab_synth.relu_activations((rows, n), 0.6, stream=n)
+    elif kind == "laplace":
+        w = dab_synth.laplace((rows, n), 0.05, stream=n)
+    elif kind == "ints":
+        w = dab_synth.small_integer_rows(rows, n, -3, 3, stream=n)
+    elif kind == "cluster":
+        w = dab_synth.two_cluster_rows(rows, n, stream=n)
+    else:
+        w = -dab_synth.relu_activations((rows, n), 0.3, stream=n)
+    w = np.ascontiguousarray(w, np.float32)
+    w[0, :] = 0.25                                   # a constant row
+    w[1, :] = 0.0                                    # a row of zeros
+    w[2, 5] = np.nan                                 # a non-finite row
+    wd = to_dev(w)
+    outs = {}
+    for coder in (dab.PATCHES_SORT, dab.PATCHES_HIST, dab.PATCHES_AUTO):
+        dab.dab_set_patch_coder(coder)
+        outs[coder] = dab.dab_binarize(wd)
+    dab.dab_set_patch_coder(dab.PATCHES_AUTO)
+    torch.cuda.synchronize()
+    s, h, au = outs[dab.PATCHES_SORT], outs[dab.PATCHES_HIST], outs[dab.PATCHES_AUTO]
+    for name in ("K", "mask", "flags"):
+        assert torch.equal(getattr(s, name), getattr(h, name)) and torch.equal(getattr(s, name), getattr(au, name)), name
+    ok = (s.flags == 0)
+    assert torch.equal(s.alpha[ok], h.alpha[ok]) and torch.equal(s.beta[ok], h.beta[ok])
+    check_coded(h, oracle.binarize(w), n, log=print)
+
+
+def test_large_dense_matrix_takes_the_histogram_search_by_default(dab):
+    # 2048 rows: the default choice runs the histogram kernel; sparse and dense rows mixed in one matrix
+    from parity_util import check_coded
+    n = 1152
+    w = np.concatenate([dab_synth.laplace((1024, n), 0.05, stream=61), dab_synth.relu_activations((1024, n), 0.6, stream=62)])
+    w = np.ascontiguousarray(w[np.argsort(dab_synth.uniform01(3, 9, 0, 2048))], np.float32)    # interleave them
+    wd = to_dev(w)
+    dab.dab_set_patch_coder(dab.PATCHES_SORT)
+    s = dab.dab_binarize(wd)
+    dab.dab_set_patch_coder(dab.PATCHES_AUTO)
+    au = dab.dab_binarize(wd)
+    torch.cuda.synchronize()
+    for name in ("K", "mask", "flags", "alpha", "beta"):
+        assert torch.equal(getattr(s, name), getattr(au, name)), name
+    sel = np.arange(0, 2048, 37)
+    sub = dab.Coded(au.mask[sel], au.K[sel], au.alpha[sel], au.beta[sel], au.flags[sel], n)
+    check_coded(sub, oracle.binarize(w[sel]), n, log=print)
