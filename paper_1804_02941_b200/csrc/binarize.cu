@@ -190,17 +190,17 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kerne
     const bool flip = res.mode == 1, none = res.mode == 2;
     const float tv = key_value(res.tkey);
     uint32_t* mrow = mask_out + row * (int64_t)ld_mask;
-    uint32_t mine = 0;
+    const bool keep = !none;
+    for (int kb = 0; kb < rounds; kb += 32) {  // 32 mask words at a time: word kb + j ends up in lane j
+      const int kend = min(32, rounds - kb);
+      uint32_t mine = 0;
 #pragma unroll 4
-    for (int k = 0; k < rounds; ++k) {
-      const float x = element(k);
-      const bool bit = !none && (k * 32 + lane < n) && ((x >= tv) != flip);
-      const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
-      if ((k & 31) == lane) mine = word;
-      if ((k & 31) == 31 || k == rounds - 1) {
-        const int w = (k & ~31) + lane;
-        if (w <= k) mrow[w] = mine;
+      for (int kk = 0; kk < kend; ++kk) {
+        const float x = element(kb + kk);
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, keep && ((kb + kk) * 32 + lane < n) && ((x >= tv) != flip));
+        if (kk == lane) mine = word;
       }
+      if (lane < kend) mrow[kb + lane] = mine;
     }
     for (int w = rounds + lane; w < ld_mask; w += 32) mrow[w] = 0u;
   }
