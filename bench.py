@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"],
                     help="contraction kernel: auto (tensor cores except on tiny problems; every layer of this workload takes "
                          "them), tensor (forced) or popc (AND + population counts)")
-    ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist"],
+    ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist", "pixel"],
                     help="patch coder: auto (by tile density), sort (full sort per patch) or hist (histogram-pruned search)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
@@ -256,7 +256,7 @@ def run_dab(args):
         dist.init_process_group("nccl", device_id=dev)
     dab.lib()
     dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
-    dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST}[args.patch_coder])
+    dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST, "pixel": dab.PATCHES_PIXEL}[args.patch_coder])
     hbm_peak, peak_src, sm_max_mhz = load_peaks()
 
     layers = select_layers(configs.config5(args.batch), args)

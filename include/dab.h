@@ -300,7 +300,7 @@ dab_contraction dab_get_contraction(void);
  *                      values and hand the others (above about 45 % non-zero) to the histogram coder.
  * Process-wide, read at each call.
  */
-typedef enum { DAB_PATCHES_AUTO = 0, DAB_PATCHES_SORT = 1, DAB_PATCHES_HIST = 2 } dab_patch_coder;
+typedef enum { DAB_PATCHES_AUTO = 0, DAB_PATCHES_SORT = 1, DAB_PATCHES_HIST = 2, DAB_PATCHES_PIXEL = 3 } dab_patch_coder;
 dab_status dab_set_patch_coder(dab_patch_coder coder);
 dab_patch_coder dab_get_patch_coder(void);
 

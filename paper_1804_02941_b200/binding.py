@@ -410,7 +410,7 @@ def dab_set_contraction(path: int) -> None:
     _check(lib().dab_set_contraction(int(path)), "dab_set_contraction")
 
 
-PATCHES_AUTO, PATCHES_SORT, PATCHES_HIST = 0, 1, 2
+PATCHES_AUTO, PATCHES_SORT, PATCHES_HIST, PATCHES_PIXEL = 0, 1, 2, 3
 
 
 def dab_set_patch_coder(coder: int) -> None:

@@ -433,7 +433,8 @@ dab_status dab_set_contraction(dab_contraction path) {
 }
 
 dab_status dab_set_patch_coder(dab_patch_coder coder) {
-  if (coder != DAB_PATCHES_AUTO && coder != DAB_PATCHES_SORT && coder != DAB_PATCHES_HIST) return DAB_ERR_INVALID_ARG;
+  if (coder != DAB_PATCHES_AUTO && coder != DAB_PATCHES_SORT && coder != DAB_PATCHES_HIST && coder != DAB_PATCHES_PIXEL)
+    return DAB_ERR_INVALID_ARG;
   set_patch_coder_mode((int)coder);
   return DAB_OK;
 }

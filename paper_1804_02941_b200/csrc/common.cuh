@@ -91,7 +91,13 @@ cudaError_t read_mma_wait_timeouts(unsigned int* count);
 cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x, int32_t* pK,
                                     float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp, uint32_t* pflags,
                                     cudaStream_t stream);
-// Patch coder selection: 0 by tile density (default), 1 sort-based only, 2 histogram-pruned wherever it applies.
+// Pixel-histogram patch coder (pixhist.cu): per-pixel bucket tables shared by the overlapping patches of a tile,
+// then the full-sort kernel on the patches it marked.  *applicable = false: nothing was launched (no tile fits).
+cudaError_t launch_binarize_patches_pixhist(const dab_conv_desc& d, int32_t Ho, int32_t Wo, const float* x,
+                                            int32_t* pK, float* pgamma, float* pdelta, uint32_t* pmask, int32_t ldp,
+                                            uint32_t* pflags, cudaStream_t stream, bool* applicable);
+// Patch coder selection: 0 default, 1 sort-based only, 2 histogram-pruned per patch wherever it applies,
+// 3 pixel-histogram coder wherever it applies.
 int patch_coder_mode();
 void set_patch_coder_mode(int mode);
 // Two flag words for a chain of kernels of one call (see PatchArgs in patches.cu) and the call's id.

@@ -655,6 +655,11 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
   const int mode = patch_coder_mode();
   cudaError_t e;
+  if (mode == 3) {
+    bool applicable = false;
+    e = launch_binarize_patches_pixhist(d, Ho, Wo, x, pK, pgamma, pdelta, pmask, ldp, pflags, stream, &applicable);
+    if (e != cudaSuccess || applicable) return e;
+  }
   if (mode == 1 || a.n > 8192) {
     // Sort-based coders only.  The patch lengths of the common 3x3 layers (576 values per warp) have variants
     // without bounds tests whose group size suits rows that are at least half zeros.

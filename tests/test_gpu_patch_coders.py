@@ -74,8 +74,9 @@ def test_histogram_coder_equals_sort_coder_and_checker(dab, ci):
     a = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_SORT)
     b = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_HIST)
     c = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_AUTO)
-    for s, h, au in zip(a, b, c):
-        assert torch.equal(s, h) and torch.equal(s, au)
+    px = _code(dab, xd, C, kh, kw, stride, pad, dab.PATCHES_PIXEL)
+    for s, h, au, pp in zip(a, b, c, px):
+        assert torch.equal(s, h) and torch.equal(s, au) and torch.equal(s, pp)
     n = C * kh * kw
     rows = oracle.im2col(x, kh, kw, stride, pad)
     sel = np.unique(np.concatenate([[0, len(rows) - 1], (dab_synth.uniform01(96, ci, 0, 64) * len(rows)).astype(np.int64)]))
@@ -95,6 +96,8 @@ def test_nonfinite_tiles_fall_back(dab):
     a = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
     b = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_HIST)
     c = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
+    px = _code(dab, xd, 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_PIXEL)
+    assert torch.equal(a[0], px[0]) and torch.equal(a[3], px[3]) and torch.equal(a[4], px[4])
     assert torch.equal(a[0], b[0]) and torch.equal(a[3], b[3]) and torch.equal(a[4], b[4])
     assert torch.equal(a[0], c[0]) and torch.equal(a[3], c[3]) and torch.equal(a[4], c[4])
     assert int((b[4] == 2).sum()) == 9 + 4
@@ -108,8 +111,9 @@ def test_mixed_density_batches_split_between_the_coders(dab):
     xd = to_dev(x)
     a = _code(dab, xd, 128, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
     c = _code(dab, xd, 128, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
-    for s, au in zip(a, c):
-        assert torch.equal(s, au)
+    px = _code(dab, xd, 128, 3, 3, (1, 1), (1, 1), dab.PATCHES_PIXEL)
+    for s, au, pp in zip(a, c, px):
+        assert torch.equal(s, au) and torch.equal(s, pp)
     x64 = np.ascontiguousarray(x[:, :64])
     a = _code(dab, to_dev(x64), 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
     c = _code(dab, to_dev(x64), 64, 3, 3, (1, 1), (1, 1), dab.PATCHES_AUTO)
