@@ -28,7 +28,8 @@ namespace {
 
 constexpr int kFixWarps = 8;      // warps of the kernel that sorts the marked patches
 constexpr int kFixThreads = kFixWarps * 32;
-constexpr int kHullCap = 256;   // values the exact search takes at most (8 per lane)
+constexpr int kHullCap = 256;        // values the exact search takes at most from the per-warp scratch array (8 per lane)
+constexpr int kHullCapRegs = 1024;   // the same when the hull goes straight into registers (3 x 3 windows; 32 per lane)
 
 struct PixArgs {
   dab_conv_desc d;
@@ -354,39 +355,50 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
           neg = __shfl_sync(0xFFFFFFFFu, tn, 31);
           Pneg = __shfl_sync(0xFFFFFFFFu, tp, 31);
         }
-        float best = -1.0f;
-        float bound[BPL];
+        // objective at the upper edge of every bucket (empty ones repeat their neighbour's split) and at the split
+        // after the run of zeros; a bucket's lower edge is the upper edge of the bucket before it, except for the
+        // first positive bucket, whose lower edge is the split after the zeros
+        const float dz1 = (z > 0 && neg + z < a.n) ? objective_bound((double)(neg + z), Pneg, T, nd) : -1.0f;
+        float best = dz1;
+        float e1[BPL], bound[BPL];
+#pragma unroll
+        for (int j = 0; j < BPL; ++j) {
+          const int b = j * 32 + lane;
+          const int s1 = cc[j] + (b >= qz.B0 ? z : 0);
+          e1[j] = (s1 > 0 && s1 < a.n) ? objective_bound((double)s1, cs[j], T, nd) : -1.0f;
+          best = fmaxf(best, e1[j]);
+        }
+        float dz0 = -1.0f;  // the split before the zeros = upper edge of the last negative bucket
+        if (qz.B0 > 0) {
+          const int jn = (qz.B0 - 1) >> 5;
+          float t = -1.0f;
+#pragma unroll
+          for (int j = 0; j < BPL; ++j)
+            if (j == jn) t = e1[j];
+          t = __shfl_sync(0xFFFFFFFFu, t, 31);
+          if (z > 0) dz0 = t;
+        }
 #pragma unroll
         for (int j = 0; j < BPL; ++j) {
           const int b = j * 32 + lane;
           const int c = cc[j] - pc[j];
-          const int zadd = b >= qz.B0 ? z : 0;
-          const int s0 = pc[j] + zadd, s1 = cc[j] + zadd;
-          float d0 = -1.0f, d1 = -1.0f, dk = -1.0f;
-          if (c > 0) {
-            if (s0 > 0 && s0 < a.n) d0 = objective_bound((double)s0, ps[j], T, nd);
-            if (s1 > 0 && s1 < a.n) d1 = objective_bound((double)s1, cs[j], T, nd);
-            if (c >= 2) {
-              // value bounds of the bucket and the two inner corners of the region (s, P) can visit inside it
-              const double vlo = (double)(b - qz.B0) * qz.width, vhi = vlo + qz.width;
-              const double cd = (double)c, S = cs[j] - ps[j];
-              double jl = (cd * vhi - S) * qz.inv_width;
-              jl = fmin(fmax(jl, 0.0), cd);
-              const double ju = cd - jl;
-              dk = fmaxf(objective_bound((double)s0 + jl, ps[j] + jl * vlo, T, nd),
-                         objective_bound((double)s0 + ju, ps[j] + ju * vhi, T, nd));
-            }
+          const float up = __shfl_up_sync(0xFFFFFFFFu, e1[j], 1);
+          const float wrap = j ? __shfl_sync(0xFFFFFFFFu, e1[j ? j - 1 : 0], 31) : -1.0f;
+          const float d0 = (b == qz.B0 && z > 0) ? dz1 : (lane ? up : wrap);
+          float dk = -1.0f;
+          if (c >= 2) {
+            // value bounds of the bucket and the two inner corners of the region (s, P) can visit inside it
+            const int s0 = pc[j] + (b >= qz.B0 ? z : 0);
+            const double vlo = (double)(b - qz.B0) * qz.width, vhi = vlo + qz.width;
+            const double cd = (double)c, S = cs[j] - ps[j];
+            double jl = (cd * vhi - S) * qz.inv_width;
+            jl = fmin(fmax(jl, 0.0), cd);
+            const double ju = cd - jl;
+            dk = fmaxf(objective_bound((double)s0 + jl, ps[j] + jl * vlo, T, nd),
+                       objective_bound((double)s0 + ju, ps[j] + ju * vhi, T, nd));
           }
-          best = fmaxf(best, fmaxf(d0, d1));
-          bound[j] = c > 0 ? fmaxf(fmaxf(d0, d1), dk) : -2.0f;
+          bound[j] = c > 0 ? fmaxf(fmaxf(d0, e1[j]), dk) : -2.0f;
         }
-        // the two splits around the run of zeros
-        float dz0 = -1.0f, dz1 = -1.0f;
-        if (z > 0) {
-          if (neg > 0) dz0 = objective_bound((double)neg, Pneg, T, nd);
-          if (neg + z < a.n) dz1 = objective_bound((double)(neg + z), Pneg, T, nd);
-        }
-        best = fmaxf(best, fmaxf(dz0, dz1));
         best = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fmaxf(best, 0.0f))));
         const float need = best * prune_margin;
         int seg_lo = 1 << 20, seg_hi = -1;  // segments: buckets below B0 keep their index, the zeros are B0, the rest + 1
@@ -422,7 +434,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
           const double P_upto = __shfl_sync(0xFFFFFFFFu, q1, b_hi & 31);
           const int m_sub = c_upto - c_below;
           const int s_below = c_below + (seg_lo > qz.B0 ? z : 0);  // the zeros lie below the hull
-          if (m_sub < 1 || m_sub > kHullCap || (z == 0 && m_sub == a.n)) {
+          if (m_sub < 1 || m_sub > (KHW ? kHullCapRegs : kHullCap) || (z == 0 && m_sub == a.n)) {
             retry = true;
           } else {
             // ---- gather the hull (raw bits) from the ordered lists of the window's pixels ----
@@ -452,8 +464,12 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
                 res = pix_gather_sort_select<2, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
               } else if (m_sub <= 128) {
                 res = pix_gather_sort_select<4, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
-              } else {
+              } else if (m_sub <= 256) {
                 res = pix_gather_sort_select<8, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
+              } else if (m_sub <= 512) {
+                res = pix_gather_sort_select<16, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
+              } else {
+                res = pix_gather_sort_select<32, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
               }
             } else {
               int fill = 0;
@@ -504,6 +520,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
         // The lanes whose bits start in the same word form a run of 3 or 4 lanes: an OR over the run gives that
         // word's own bits, a second OR the bits that spill into the next word.
         const int groups = (C + 31) >> 5;
+#pragma unroll 2
         for (int g = 0; g < groups; ++g) {
           const int c = g * 32 + lane;
           const bool live = c < C && !none;
