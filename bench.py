@@ -24,16 +24,34 @@ UNIT = "TOPS-equiv (2*M*N*n binary ops per second / 1e12)"
 L2_BYTES = 126 * 1024 * 1024
 POPC_PER_CLK_PER_SM = 16          # integer population counts per clock per SM
 WORDS_PER_POPC = 1.5              # the contraction compresses 3 AND-ed words into 2 population counts
-SM_COUNT = 148
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the patch-coder launches of each layer at batch 256, from one
-# ncu capture of this benchmark (profiles/binarize_patches_dram_traffic_config5.md).  Valid for the kernels as
-# they were then: reset to {} when the patch coder changes.
-PATCH_CODER_DRAM_BYTES = {"l1_0": 275064576, "l1_1": 271620608, "l1_2": 272581632, "l1_3": 272041216, "l2_0":
-                          222675712, "l2_1": 119762688, "l2_2": 120052736, "l2_3": 119627776, "l3_0": 106836736,
-                          "l3_1": 52807680, "l3_2": 53128448, "l3_3": 52924928, "l4_0": 52207872, "l4_1": 26969344,
-                          "l4_2": 26978816, "l4_3": 26957568}
+# Sources of the patch coder: a measured DRAM-traffic record is only quoted while these files are unchanged.
+PATCH_CODER_SOURCES = ("pixhist.cu", "patches.cu", "rowcode.cuh", "histcode.cuh", "common.cuh")
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "patch_coder_dram_traffic.json")
+
+
+def patch_coder_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in PATCH_CODER_SOURCES:
+        with open(os.path.join(ROOT, "paper_1804_02941_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_patch_coder_traffic(layer_names, batch, dense):
+    """Average DRAM bytes per patch-coder launch from the committed profiler record, or None when there is no record
+    for this workload or the kernels have changed since it was taken."""
+    try:
+        with open(TRAFFIC_RECORD) as f:
+            rec = json.load(f)
+        if rec.get("source_sha256") != patch_coder_source_hash() or rec.get("batch") != batch or bool(rec.get("dense")) != bool(dense):
+            return None
+        per_layer = rec["dram_bytes_per_launch"]
+        return sum(per_layer[n] for n in layer_names) / len(layer_names)
+    except (OSError, KeyError, ValueError):
+        return None
 
 
 def parse_args():
@@ -50,8 +68,9 @@ def parse_args():
                     help="contraction kernel: auto (tensor cores except on tiny problems; every layer of this workload takes "
                          "them), tensor (forced) or popc (AND + population counts)")
     ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist", "pixel"],
-                    help="patch coder: auto (by tile density), sort (full sort per patch) or hist (histogram-pruned search)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+                    help="patch coder: auto (pixel-histogram coder wherever patches overlap), sort (full sort per patch), "
+                         "hist (histogram-pruned search per patch) or pixel (pixel-histogram coder wherever it applies)")
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -206,10 +225,14 @@ def run_reference(args):
     }))
 
 
-def patch_launches(n, coder):
-    """Kernels one dab_binarize_patches call launches (some end at once when no tile was handed to them)."""
+def patch_launches(L, coder):
+    """Kernels one dab_binarize_patches call launches (some end at once when nothing was handed to them)."""
+    n = L.n
     if n <= 256:
         return 1
+    pixel = n <= 8192 and L.kh * L.kw >= 4 and L.patches >= 1024 and not (L.stride * L.stride >= 4 and L.C > 128)
+    if coder == "pixel" or (coder == "auto" and pixel):
+        return 2                      # pixel-histogram coder, then the kernel that sorts the patches it marked
     if coder == "auto":
         return 3                      # sort-based coder, histogram coder on the dense tiles, group kernel on the rest
     if coder == "hist":
@@ -258,6 +281,7 @@ def run_dab(args):
     dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
     dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST, "pixel": dab.PATCHES_PIXEL}[args.patch_coder])
     hbm_peak, peak_src, sm_max_mhz = load_peaks()
+    SM_COUNT = torch.cuda.get_device_properties(dev).multi_processor_count
 
     layers = select_layers(configs.config5(args.batch), args)
     # one host tensor per distinct input shape (pinned: it is also the source of the end-to-end copies);
@@ -345,13 +369,13 @@ def run_dab(args):
     # (4*ceil(n/32) B) and K, gamma, delta (12 B) written
     patch_bytes = sum(4 * L.N * L.C * L.H * L.W + L.patches * (4 * dab.dab_words_per_row(L.n) + 12) for L in layers)
     binarize_gbs = patch_bytes * args.steps / (k_ms["binarize_patches"] * 1e-3) / 1e9
-    traffic = None
-    if args.batch == 256 and not args.dense and all(L.name in PATCH_CODER_DRAM_BYTES for L in layers):
-        traffic = sum(PATCH_CODER_DRAM_BYTES[L.name] for L in layers) / len(layers)   # per layer launch, like achieved
-    roofline = {"kernel": "binarize_patches_{warp,group}_kernel", "bound": "hbm", "achieved": binarize_gbs,
+    traffic = measured_patch_coder_traffic([L.name for L in layers], args.batch, args.dense) if args.patch_coder == "auto" else None
+    roofline = {"kernel": "binarize_patches_pixhist_kernel (+ binarize_patches_fixup_kernel; strided 256-channel layers: "
+                          "binarize_patches_group_kernel)", "bound": "hbm", "achieved": binarize_gbs,
                 "peak": hbm_peak, "unit": "GB/s", "frac": binarize_gbs / hbm_peak, "traffic": traffic,
-                "traffic_note": "measured DRAM bytes per layer launch (ncu), average over the layers; algorithmic "
-                                "average alongside", "peak_source": peak_src,
+                "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum per layer launch, average over the layers, from "
+                                "profiles/patch_coder_dram_traffic.json; null when the coder's sources have changed since "
+                                "that capture", "peak_source": peak_src,
                 "algorithmic_bytes_per_launch_avg": patch_bytes / len(layers),
                 "avg_launch_ms": k_ms["binarize_patches"] / launches_per_kind,
                 "share_of_step": k_ms["binarize_patches"] / sum(k_ms.values())}
@@ -377,6 +401,10 @@ def run_dab(args):
         int8_peak, int8_src = load_int8_peak()
         roofline_contract = {"kernel": "binary_gemm_mma_kernel", "bound": "tensor", "peak": int8_peak,
                              "frac": contract_tops / int8_peak, "peak_source": int8_src,
+                             "popc_bound": popc_peak_derived, "frac_of_popc_bound": contract_tops / popc_peak_derived,
+                             "popc_bound_source": "the integer-pipe bound of the population-count kernel (16 popc/clk/SM x "
+                                                  "1.5 words per popc x SMs x max clock x 64): what the same contraction "
+                                                  "could reach without tensor cores",
                              "note": "kind::i8 on 0/1 bytes; the kernel's time goes to expanding mask words to bytes, the fp64 "
                                      "rescale of every count and the output store, not to the tensor pipe", **common}
     else:
@@ -455,7 +483,7 @@ def run_dab(args):
                "scaling": "weak", "vs_baseline": None, "dtype": "u8 x u8 -> s32 tensor-core counts + f64 objective/rescale" if args.contraction != "popc"
                else "u32 popcount + f64 objective/rescale",
                "data": "synthetic", "config": workload_config(args), "clocks": clocks, "e2e": e2e,
-               "gpu_launches": (2 * len(layers) + sum(patch_launches(L.n, args.patch_coder) for L in layers)) * args.steps,
+               "gpu_launches": (2 * len(layers) + sum(patch_launches(L, args.patch_coder) for L in layers)) * args.steps,
                "kernel_ms_per_step": {k: v / args.steps for k, v in k_ms.items()},
                "binarize_gbs": binarize_gbs, "roofline": roofline, "roofline_contraction": roofline_contract,
                "wbin": wbin, "cpu_baseline": cpu_baseline, "contraction_wait_failures": dab.dab_contraction_wait_failures()}

@@ -42,8 +42,11 @@ size_t dab_binary_conv_static_capacity(void) { return kStaticScratchBytes; }
 dab_status dab_binary_conv_static(const dab_conv_desc* desc, const float* d_x, const uint32_t* d_wmask, int32_t ldw,
                                   const int32_t* d_wK, const float* d_walpha, const float* d_wbeta, float* d_y,
                                   void* stream) {
+  if (!desc) return DAB_ERR_INVALID_ARG;
+  if (desc->C > 0 && desc->kh > 0 && desc->kw > 0 && (int64_t)desc->C * desc->kh * desc->kw > DAB_MAX_N)
+    return DAB_ERR_UNSUPPORTED;                            // row length beyond DAB_MAX_N, as dab_binary_conv reports it
   const size_t need = dab_binary_conv_workspace(desc);
-  if (need == 0) return DAB_ERR_INVALID_ARG;               // impossible geometry or row length beyond DAB_MAX_N
+  if (need == 0) return DAB_ERR_INVALID_ARG;               // impossible geometry
   if (need > kStaticScratchBytes) return DAB_ERR_UNSUPPORTED;  // layer too large for the built-in scratch
   void* scratch = nullptr;
   dab_status s = scratch_address(&scratch);

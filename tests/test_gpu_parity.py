@@ -236,8 +236,11 @@ def test_conv_with_sign_coded_inputs_matches_checker(dab, ci):
     assert np.array_equal(det.pK.cpu().numpy(), ref.p_K) and np.array_equal(unpack(words(det.pmask), n), ref.p_e)
     assert rel_close(det.pgamma.cpu().numpy(), ref.p_gamma).all() and rel_close(det.pdelta.cpu().numpy(), ref.p_delta).all()
     assert np.array_equal(det.p11.cpu().numpy(), ref.p_p11)
-    # gamma may differ in the last bit (summation order), so the outputs are compared within the tolerance
-    assert rel_close(y.cpu().numpy(), ref.y, 2e-5).all()
+    # gamma, delta: the fp64 sum of |x| over the row is formed in another order than the checker's; it is exact
+    # (hence equal) unless the row mixes magnitudes more than 2^29 apart, so the scales agree to the bit here and
+    # the outputs, formed from them by the same fp64 expression, meet the 1e-5 bound everywhere
+    assert np.array_equal(det.pgamma.cpu().numpy(), ref.p_gamma) and np.array_equal(det.pdelta.cpu().numpy(), ref.p_delta)
+    assert rel_close(y.cpu().numpy(), ref.y).all()
 
 
 @pytest.mark.parametrize("batch", [1, 2, 19])
