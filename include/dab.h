@@ -9,7 +9,8 @@
  *
  * Conventions for every entry point
  *   - Pointers named d_* are DEVICE pointers owned by the caller; h_* are HOST pointers.  The
- *     library allocates and frees no device memory and keeps no state between calls.
+ *     library allocates and frees no device memory.  What it keeps between calls is listed under
+ *     "State" below; none of it carries data from one call's inputs to another call's outputs.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue
  *     work on that stream and return without synchronising, except where stated.
  *   - Errors are return codes.  Arguments are validated on the host before anything is
@@ -19,6 +20,20 @@
  *     beyond n and words beyond ceil(n/32) are written as 0 by the producers and must be 0 for
  *     the consumers.
  *   - Row length limit: 1 <= n <= DAB_MAX_N.
+ *
+ * State kept by the library (process-wide unless stated; every item is safe to use from several threads)
+ *   - the patch-coder and contraction choices (dab_set_patch_coder, dab_set_contraction): atomic integers
+ *     read once at the start of each call;
+ *   - per device: the SM count and, per kernel, the largest dynamic shared-memory size it was opted in to
+ *     (caches of driver queries, behind a mutex);
+ *   - per device: two copy streams and a few events of dab_binary_conv_host, created on its first call;
+ *     calls of that entry point on one device are serialised by a lock;
+ *   - per device: the address of dab_binary_conv_static's scratch array, and the array itself, which keeps
+ *     the last call's patch codes (see that entry point);
+ *   - per device: two counters of barrier waits that ran out (dab_contraction_wait_failures).
+ *   Cached device addresses do not survive cudaDeviceReset: do not reset a device while the library is loaded.
+ *   Calls on different streams may run concurrently; kernels of one call hand work to each other only through
+ *   that call's own output arrays.
  */
 #ifndef DAB_H
 #define DAB_H
@@ -287,18 +302,27 @@ dab_status dab_set_contraction(dab_contraction path);
 dab_contraction dab_get_contraction(void);
 
 /*
- * Which kernels code the patches in dab_binarize_patches and the convolution entry points built on it
- * (Section 4.1 / Algorithm 1 per patch; every choice gives the same codes bit for bit):
- *   DAB_PATCHES_SORT   every patch is sorted in full (its exact zeros are only counted) and every split evaluated;
- *   DAB_PATCHES_HIST   patches of 257..8192 values go through a histogram of their values that bounds the
- *                      objective per bucket (it is convex in the split size and the prefix sum) and leaves only
- *                      the few buckets that can hold the maximum to the exact search; tiles it cannot settle (a
- *                      hull of more than 256 (patches of fewer than 1024 values) or 1024 values, non-finite inputs) fall to the sorting kernel.  Its cost does
- *                      not grow with the number of non-zero values: 2.5x to 6.5x faster than sorting on inputs
- *                      without zeros, about 10 % slower on inputs that are 60 % zeros;
- *   DAB_PATCHES_AUTO   (default) per tile of the input: the sorting kernels take the tiles with few non-zero
- *                      values and hand the others (above about 45 % non-zero) to the histogram coder.
- * Process-wide, read at each call.
+ * Which kernels code the patches in dab_binarize_patches and the convolution entry points built on it, and the rows
+ * in dab_binarize (Section 4.1 / Algorithm 1 per row; every choice gives the same codes bit for bit):
+ *   DAB_PATCHES_SORT   every row is sorted in full (its exact zeros are only counted) and every split evaluated;
+ *   DAB_PATCHES_PIXEL  patches of 257..8192 values: the values of every input pixel (its C channels) are counted once
+ *                      per tile into buckets of power-of-two width, with exact fp64 sums; a patch adds the tables of
+ *                      its kh*kw pixels, which gives the split size and prefix sum at every bucket edge exactly.  The
+ *                      objective is convex in (split size, prefix sum), so inside a bucket it is bounded by its values
+ *                      at the corners of the region the bucket's count, sum and value bounds allow; only the few
+ *                      buckets whose bound reaches the best edge value are searched exactly.  Work per pixel is
+ *                      shared by the up to kh*kw patches that contain it.  Patches it cannot settle (a hull of more
+ *                      than 1024 values, a constant row without zeros, magnitudes outside 2^-40..2^40, a NaN or an
+ *                      infinity in the tile) are sorted in full by a second kernel;
+ *   DAB_PATCHES_HIST   rows and patches of 257..8192 values, one warp each: a histogram of the row's own values
+ *                      quantised to 24 bits of its range, the same bound per bucket with a margin for the
+ *                      quantisation, exact search of what survives; rows it cannot settle fall to the sorting kernel;
+ *   DAB_PATCHES_AUTO   (default) patches: DAB_PATCHES_PIXEL wherever a patch spans several pixels and the layer has
+ *                      at least 1024 patches (except strided windows over more than 128 channels, which overlap too
+ *                      little); otherwise per tile of the input the sorting kernels for tiles with few non-zero values
+ *                      and DAB_PATCHES_HIST for the others.  Rows of a matrix: DAB_PATCHES_HIST from 2048 rows on,
+ *                      DAB_PATCHES_SORT below.
+ * Process-wide, read once at the start of each call.
  */
 typedef enum { DAB_PATCHES_AUTO = 0, DAB_PATCHES_SORT = 1, DAB_PATCHES_HIST = 2, DAB_PATCHES_PIXEL = 3 } dab_patch_coder;
 dab_status dab_set_patch_coder(dab_patch_coder coder);
@@ -311,15 +335,6 @@ dab_patch_coder dab_get_patch_coder(void);
  * pointer).  Synchronises the device.  0 on every correct run.
  */
 dab_status dab_contraction_wait_failures(uint32_t* h_count);
-
-/*
- * dab_popc_probe — measurement aid, not part of the method: runs `iters` rounds of independent
- * AND + population-count + add chains in every thread of a grid of `blocks` x 256 threads and
- * writes one word per thread to d_sink (blocks*256 words), so that a caller timing it obtains the
- * device's achievable rate for the inner operation of dab_binary_gemm.
- * Word operations executed = blocks * 256 * iters * 16.
- */
-dab_status dab_popc_probe(uint32_t* d_sink, int32_t blocks, int32_t iters, void* stream);
 
 #ifdef __cplusplus
 }

@@ -111,6 +111,52 @@ def _dev(t, dtype, name):
     return t
 
 
+# ------------------------------------------------------------------------------------------------------------
+# Output allocation.  With guards switched on (the GPU tests do this), every output tensor this module creates sits
+# between two 256-byte guard zones filled with a pattern; guards_check() verifies that no kernel wrote into them.
+# It stands in for a memory checker: it catches writes just before or behind an output, not every stray access.
+# ------------------------------------------------------------------------------------------------------------
+_GUARD = 256
+_GUARD_BYTE = 0xA5
+_guards_on = False
+_guarded = []
+
+
+def guards_enable(on: bool) -> None:
+    global _guards_on
+    _guards_on = bool(on)
+    if not on:
+        _guarded.clear()
+
+
+def _new(shape, dtype, device):
+    if not _guards_on:
+        return torch.empty(shape, dtype=dtype, device=device)
+    if isinstance(shape, int):
+        shape = (shape,)
+    numel = 1
+    for d in shape:
+        numel *= int(d)
+    nbytes = numel * torch.empty((), dtype=dtype).element_size()
+    pad = (-nbytes) % 16
+    raw = torch.full((_GUARD + nbytes + pad + _GUARD,), _GUARD_BYTE, dtype=torch.uint8, device=device)
+    _guarded.append((raw, nbytes))
+    return raw[_GUARD:_GUARD + nbytes].view(dtype).view(tuple(int(d) for d in shape))
+
+
+def guards_check() -> int:
+    """Verifies the guard zones of every tensor handed out since the last check; returns how many were checked."""
+    torch.cuda.synchronize()
+    n = len(_guarded)
+    for raw, nbytes in _guarded:
+        front, back = raw[:_GUARD], raw[_GUARD + nbytes:]
+        if not (bool((front == _GUARD_BYTE).all()) and bool((back == _GUARD_BYTE).all())):
+            _guarded.clear()
+            raise AssertionError("a kernel wrote outside an output tensor of %d bytes" % nbytes)
+    _guarded.clear()
+    return n
+
+
 def dab_words_per_row(n: int) -> int:
     return int(lib().dab_words_per_row(C.c_int32(n)))
 
@@ -147,9 +193,9 @@ def dab_binarize(values: torch.Tensor, ld_mask: int | None = None, stream=None, 
     rows, n = values.shape
     ld = dab_default_ld(n) if ld_mask is None else ld_mask
     dev = values.device
-    out = Coded(torch.empty((rows, ld), dtype=torch.int32, device=dev), torch.empty(rows, dtype=torch.int32, device=dev),
-                torch.empty(rows, dtype=torch.float32, device=dev), torch.empty(rows, dtype=torch.float32, device=dev),
-                torch.empty(rows, dtype=torch.int32, device=dev), n)
+    out = Coded(_new((rows, ld), torch.int32, dev), _new(rows, torch.int32, dev),
+                _new(rows, torch.float32, dev), _new(rows, torch.float32, dev),
+                _new(rows, torch.int32, dev), n)
     ldv = values.stride(0) if rows > 1 else max(n, values.stride(0))
     st = getattr(lib(), _entry)(_ptr(values), rows, n, ldv, _ptr(out.K), _ptr(out.alpha), _ptr(out.beta),
                                 _ptr(out.mask), ld, _ptr(out.flags), _stream(stream))
@@ -173,8 +219,8 @@ def dab_pack(bits: torch.Tensor, ld_mask: int | None = None, stream=None):
         raise ValueError("bits must be 2-D with unit inner stride")
     rows, n = bits.shape
     ld = dab_default_ld(n) if ld_mask is None else ld_mask
-    mask = torch.empty((rows, ld), dtype=torch.int32, device=bits.device)
-    K = torch.empty(rows, dtype=torch.int32, device=bits.device)
+    mask = _new((rows, ld), torch.int32, bits.device)
+    K = _new(rows, torch.int32, bits.device)
     ldb = bits.stride(0) if rows > 1 else max(n, bits.stride(0))
     _check(lib().dab_pack(_ptr(bits), rows, n, ldb, _ptr(mask), ld, _ptr(K), _stream(stream)), "dab_pack")
     return mask, K
@@ -186,8 +232,8 @@ def dab_binary_gemm(a: Coded, b: Coded, want_p11: bool = False, out: torch.Tenso
         raise ValueError("row lengths differ")
     M, N = a.mask.shape[0], b.mask.shape[0]
     dev = a.mask.device
-    Cm = torch.empty((M, N), dtype=torch.float32, device=dev) if out is None else out
-    p11 = torch.empty((M, N), dtype=torch.int32, device=dev) if want_p11 else None
+    Cm = _new((M, N), torch.float32, dev) if out is None else out
+    p11 = _new((M, N), torch.int32, dev) if want_p11 else None
     st = lib().dab_binary_gemm(M, N, a.n, _ptr(a.mask), a.ld, _ptr(a.K), _ptr(a.alpha), _ptr(a.beta), _ptr(b.mask),
                                b.ld, _ptr(b.K), _ptr(b.alpha), _ptr(b.beta), _ptr(Cm), Cm.stride(0) if M > 1 else max(N, 1),
                                _ptr(p11), N, _stream(stream))
@@ -239,18 +285,18 @@ def dab_binary_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), 
     Ho, Wo = dab_conv_output_size(desc)
     dev = x.device
     if y is None:
-        y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=dev)
+        y = _new((x.shape[0], Cout, Ho, Wo), torch.float32, dev)
     need = dab_binary_conv_workspace(desc)
     if workspace is None:
-        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+        workspace = _new(need, torch.uint8, dev)
     det = None
     if details:
         P = x.shape[0] * Ho * Wo
-        det = ConvDetails(torch.empty(P, dtype=torch.int32, device=dev), torch.empty(P, dtype=torch.float32, device=dev),
-                          torch.empty(P, dtype=torch.float32, device=dev),
-                          torch.empty((P, dab_default_ld(w.n)), dtype=torch.int32, device=dev),
-                          torch.empty(P, dtype=torch.int32, device=dev),
-                          torch.empty((P, Cout), dtype=torch.int32, device=dev))
+        det = ConvDetails(_new(P, torch.int32, dev), _new(P, torch.float32, dev),
+                          _new(P, torch.float32, dev),
+                          _new((P, dab_default_ld(w.n)), torch.int32, dev),
+                          _new(P, torch.int32, dev),
+                          _new((P, Cout), torch.int32, dev))
     entry = lib().dab_binary_conv_sign if sign_inputs else lib().dab_binary_conv
     st = entry(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha), _ptr(w.beta),
                                _ptr(y), _ptr(workspace), workspace.numel(),
@@ -301,7 +347,7 @@ def dab_binary_conv_host(x_host: torch.Tensor, w: Coded, kh: int, kw: int, strid
     if workspace is None:
         if not wait:
             raise ValueError("wait=False needs a caller-owned workspace that outlives the queued work")
-        workspace = torch.empty(need, dtype=torch.uint8, device=w.mask.device)
+        workspace = _new(need, torch.uint8, w.mask.device)
     fn = lib().dab_binary_conv_host if wait else lib().dab_binary_conv_host_async
     st = fn(C.byref(desc), C.c_void_p(x_host.data_ptr()), _ptr(w.mask), w.ld, _ptr(w.K),
                                     _ptr(w.alpha), _ptr(w.beta), C.c_void_p(y_host.data_ptr()), _ptr(workspace),
@@ -331,7 +377,7 @@ def dab_binary_conv_static(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(
     desc = make_desc(tuple(x.shape), Cout, kh, kw, stride, pad)
     Ho, Wo = dab_conv_output_size(desc)
     if y is None:
-        y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=x.device)
+        y = _new((x.shape[0], Cout, Ho, Wo), torch.float32, x.device)
     st = lib().dab_binary_conv_static(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.K), _ptr(w.alpha),
                                       _ptr(w.beta), _ptr(y), _stream(stream))
     _check(st, "dab_binary_conv_static")
@@ -352,10 +398,10 @@ def dab_wbin_conv(x: torch.Tensor, w: Coded, kh: int, kw: int, stride=(1, 1), pa
     desc = make_desc(tuple(x.shape), Cout, kh, kw, stride, pad)
     Ho, Wo = dab_conv_output_size(desc)
     if y is None:
-        y = torch.empty((x.shape[0], Cout, Ho, Wo), dtype=torch.float32, device=x.device)
+        y = _new((x.shape[0], Cout, Ho, Wo), torch.float32, x.device)
     need = dab_wbin_conv_workspace(desc)
     if workspace is None:
-        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        workspace = _new(need, torch.uint8, x.device)
     st = lib().dab_wbin_conv(C.byref(desc), _ptr(x), _ptr(w.mask), w.ld, _ptr(w.alpha), _ptr(w.beta), _ptr(y),
                              _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "dab_wbin_conv")
@@ -370,11 +416,11 @@ def dab_binarize_train(W: torch.Tensor, want_dense: bool = True, stream=None):
     rows, n = W.shape
     ld = dab_default_ld(n)
     dev = W.device
-    Wc = torch.empty((rows, n), dtype=torch.float32, device=dev)
-    Wt = torch.empty((rows, n), dtype=torch.float32, device=dev) if want_dense else None
-    out = Coded(torch.empty((rows, ld), dtype=torch.int32, device=dev), torch.empty(rows, dtype=torch.int32, device=dev),
-                torch.empty(rows, dtype=torch.float32, device=dev), torch.empty(rows, dtype=torch.float32, device=dev),
-                torch.empty(rows, dtype=torch.int32, device=dev), n)
+    Wc = _new((rows, n), torch.float32, dev)
+    Wt = _new((rows, n), torch.float32, dev) if want_dense else None
+    out = Coded(_new((rows, ld), torch.int32, dev), _new(rows, torch.int32, dev),
+                _new(rows, torch.float32, dev), _new(rows, torch.float32, dev),
+                _new(rows, torch.int32, dev), n)
     st = lib().dab_binarize_train(_ptr(W), rows, n, W.stride(0) if rows > 1 else n, _ptr(Wc), n, _ptr(Wt), n, _ptr(out.K),
                                   _ptr(out.alpha), _ptr(out.beta), _ptr(out.mask), ld, _ptr(out.flags), _stream(stream))
     _check(st, "dab_binarize_train")
@@ -388,7 +434,7 @@ def dab_binarize_backward(Wc: torch.Tensor, coded: Coded, grad_Wt: torch.Tensor,
     rows, n = Wc.shape
     if not (Wc.is_contiguous() and grad_Wt.is_contiguous() and grad_Wt.shape == Wc.shape):
         raise ValueError("Wc and grad_Wt must be contiguous and of one shape")
-    gW = torch.empty_like(Wc)
+    gW = _new(tuple(Wc.shape), Wc.dtype, Wc.device)
     st = lib().dab_binarize_backward(_ptr(Wc), rows, n, n, _ptr(coded.mask), coded.ld, _ptr(coded.K), _ptr(grad_Wt), n,
                                      _ptr(gW), n, _stream(stream))
     _check(st, "dab_binarize_backward")
@@ -414,7 +460,8 @@ PATCHES_AUTO, PATCHES_SORT, PATCHES_HIST, PATCHES_PIXEL = 0, 1, 2, 3
 
 
 def dab_set_patch_coder(coder: int) -> None:
-    """PATCHES_AUTO (default: by tile density), PATCHES_SORT (full sort per patch) or PATCHES_HIST (histogram-pruned search)."""
+    """PATCHES_AUTO (default), PATCHES_SORT (full sort per row), PATCHES_HIST (histogram-pruned search per row) or
+    PATCHES_PIXEL (per-pixel histograms shared by overlapping patches); see include/dab.h."""
     _check(lib().dab_set_patch_coder(int(coder)), "dab_set_patch_coder")
 
 

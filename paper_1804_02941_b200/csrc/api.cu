@@ -1,5 +1,5 @@
-// C ABI of libdab: argument validation on the host, then launches.  No device memory is allocated; the only
-// state kept is the pair of copy streams of the host-buffer convolution.
+// C ABI of libdab: argument validation on the host, then launches.  No device memory is allocated; the state the
+// library keeps is listed in include/dab.h.
 #include <atomic>
 #include <mutex>
 
@@ -25,7 +25,7 @@ cudaError_t contract(const GemmArgs& g, bool lanes_along_rows, cudaStream_t stre
   const int64_t lane_rows = lanes_along_rows ? g.M : g.N, column_rows = lanes_along_rows ? g.N : g.M;
   const int mode = g_contraction.load(std::memory_order_relaxed);
   bool tensor = mode != (int)DAB_CONTRACT_POPC && column_rows <= (int64_t)65535 * 64;
-  if (mode == (int)DAB_CONTRACT_AUTO && ((lane_rows + 127) / 128) * ((column_rows + 63) / 64) < 148) tensor = false;
+  if (mode == (int)DAB_CONTRACT_AUTO && ((lane_rows + 127) / 128) * ((column_rows + 63) / 64) < sm_count()) tensor = false;
   return tensor ? launch_gemm_mma(g, lanes_along_rows, stream) : launch_gemm(g, lanes_along_rows, stream);
 }
 
@@ -505,9 +505,5 @@ dab_status dab_binarize_backward(const float* d_Wc, int64_t rows, int32_t n, int
                                          ld_grad_W, static_cast<cudaStream_t>(stream)));
 }
 
-dab_status dab_popc_probe(uint32_t* d_sink, int32_t blocks, int32_t iters, void* stream) {
-  if (!d_sink || blocks < 1 || iters < 0) return DAB_ERR_INVALID_ARG;
-  return from_cuda(launch_popc_probe(d_sink, blocks, iters, static_cast<cudaStream_t>(stream)));
-}
 
 }  // extern "C"

@@ -5,6 +5,18 @@
 
 namespace dab {
 
+// Whether any of the rows this CTA would take (row = (blockIdx.x + k * gridDim.x) * per_cta + g, g < per_cta) carries
+// the mark of an earlier kernel of the call.  Every thread of the CTA gets the same answer.
+__device__ __forceinline__ bool cta_has_marked_row(const int32_t* K_out, int64_t rows, int per_cta) {
+  int any = 0;
+  for (int64_t i = threadIdx.x;; i += blockDim.x) {
+    const int64_t row = ((int64_t)blockIdx.x + (i / per_cta) * gridDim.x) * per_cta + i % per_cta;
+    if (row >= rows) break;
+    any |= K_out[row] == kRowMark;
+  }
+  return __syncthreads_or(any) != 0;
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Rows of a matrix, one warp per row (n <= 32*R).
 // ---------------------------------------------------------------------------------------------------------
@@ -12,9 +24,10 @@ template <int R, bool kFull>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
     const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
     float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
-    uint32_t* __restrict__ flags_out, const unsigned int* marked_flag, uint32_t call_id) {
-  // marked_flag: code only the rows an earlier kernel of the call marked (K = kRowMark), and leave at once if it marked none
-  if (marked_flag && *reinterpret_cast<const volatile unsigned int*>(marked_flag) != call_id) return;
+    uint32_t* __restrict__ flags_out, int marked_only) {
+  // marked_only: code only the rows an earlier kernel of the call marked (K = kRowMark); a CTA none of whose rows is
+  // marked leaves at once
+  if (marked_only && !cta_has_marked_row(K_out, rows, kWarpsPerCta)) return;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
   uint32_t* scratch_all = reinterpret_cast<uint32_t*>(rcp + rcp_table_slots(n));
@@ -24,7 +37,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
   __syncthreads();
 
   for (int64_t row = (int64_t)blockIdx.x * kWarpsPerCta + warp; row < rows; row += (int64_t)gridDim.x * kWarpsPerCta) {
-    if (marked_flag && K_out[row] != kRowMark) continue;
+    if (marked_only && K_out[row] != kRowMark) continue;
     const float* v = values + row * ld_values;
     auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
     uint32_t kreg[R];
@@ -48,9 +61,9 @@ template <int W, int WARPS, int R, bool kFull, bool kTable>
 __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
     const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
     float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
-    uint32_t* __restrict__ flags_out, int scratch_words, const unsigned int* marked_flag, uint32_t call_id) {
-  if (marked_flag && *reinterpret_cast<const volatile unsigned int*>(marked_flag) != call_id) return;
+    uint32_t* __restrict__ flags_out, int scratch_words, int marked_only) {
   constexpr int G = WARPS / W;
+  if (marked_only && !cta_has_marked_row(K_out, rows, G)) return;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* rcp = reinterpret_cast<double*>(smem_raw);
   GroupShared* gs_all = reinterpret_cast<GroupShared*>(rcp + (kTable ? rcp_table_slots(n) : 0));
@@ -67,7 +80,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
   }
 
   for (int64_t row = (int64_t)blockIdx.x * G + group; row < rows; row += (int64_t)gridDim.x * G) {
-    if (marked_flag && K_out[row] != kRowMark) continue;  // the same for every thread of the group
+    if (marked_only && K_out[row] != kRowMark) continue;  // the same for every thread of the group
     const float* v = values + row * ld_values;
     auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
     uint32_t kreg[R];
@@ -87,32 +100,32 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
 template <int R, bool kFull>
 static cudaError_t launch_rows_warp(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                     float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                                    cudaStream_t stream, const unsigned int* marked_flag, uint32_t call_id) {
+                                    cudaStream_t stream, int marked_only) {
   auto kern = binarize_rows_warp_kernel<R, kFull>;
   size_t smem = sizeof(double) * rcp_table_slots(n) + sizeof(uint32_t) * 32 * R * kWarpsPerCta;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   int64_t blocks = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   kern<<<(unsigned)blocks, kWarpsPerCta * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask,
-                                                              ld_mask, flags, marked_flag, call_id);
+                                                              ld_mask, flags, marked_only);
   return cudaGetLastError();
 }
 
 template <int W, int WARPS, int R, bool kFull, bool kTable>
 static cudaError_t launch_rows_group(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                      float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                                     cudaStream_t stream, const unsigned int* marked_flag, uint32_t call_id) {
+                                     cudaStream_t stream, int marked_only) {
   constexpr int G = WARPS / W;
   auto kern = binarize_rows_group_kernel<W, WARPS, R, kFull, kTable>;
   int sw = scratch_words_for(n, W);
   size_t smem = (kTable ? sizeof(double) * rcp_table_slots(n) : 0) + sizeof(GroupShared) * G + sizeof(uint32_t) * (size_t)sw * G;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   int64_t blocks = (rows + G - 1) / G;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   kern<<<(unsigned)blocks, WARPS * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask,
-                                                       flags, sw, marked_flag, call_id);
+                                                       flags, sw, marked_only);
   return cudaGetLastError();
 }
 
@@ -126,7 +139,7 @@ template <int BPL>
 __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kernel(
     const float* __restrict__ values, int64_t rows, int32_t n, int64_t ld_values, int32_t* __restrict__ K_out,
     float* __restrict__ alpha_out, float* __restrict__ beta_out, uint32_t* __restrict__ mask_out, int32_t ld_mask,
-    uint32_t* __restrict__ flags_out, int min_density_pct, unsigned int* flag_out, uint32_t call_id) {
+    uint32_t* __restrict__ flags_out, int min_density_pct) {
   constexpr int B = 32 * BPL;
   constexpr int LOG2B = BPL == 1 ? 5 : BPL == 2 ? 6 : BPL == 4 ? 7 : 8;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -175,10 +188,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kerne
       retry = !hist_search<BPL>(sweep, n, qz, hist, scratch, rcp, lane, res);
     }
     if (retry) {
-      if (lane == 0) {
-        K_out[row] = kRowMark;
-        *flag_out = call_id;
-      }
+      if (lane == 0) K_out[row] = kRowMark;
       continue;
     }
     if (lane == 0) {
@@ -209,22 +219,22 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kerne
 template <int BPL>
 static cudaError_t launch_rows_hist(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                     float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                                    cudaStream_t stream, int min_density_pct, unsigned int* flag_out, uint32_t call_id) {
+                                    cudaStream_t stream, int min_density_pct) {
   auto kern = binarize_rows_hist_kernel<BPL>;
   size_t smem = sizeof(double) * rcp_table_slots(n) + (sizeof(int2) * 32 * BPL + sizeof(uint32_t) * hist_cap(BPL)) * kWarpsPerCta;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   int64_t blocks = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   kern<<<(unsigned)blocks, kWarpsPerCta * 32, smem, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask,
-                                                              ld_mask, flags, min_density_pct, flag_out, call_id);
+                                                              ld_mask, flags, min_density_pct);
   return cudaGetLastError();
 }
 
 static cudaError_t launch_rows_sort(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                                     float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
-                                    cudaStream_t stream, const unsigned int* marked_flag, uint32_t call_id) {
-#define DAB_ARGS values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, marked_flag, call_id
+                                    cudaStream_t stream, int marked_only) {
+#define DAB_ARGS values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, marked_only
   // A matrix may have few rows (a layer's filters), so a row gets enough warps for at most 8 keys per thread
   // even when none of its values is zero: short critical path per row, and the 8-key network is the most
   // efficient one per element.
@@ -246,18 +256,15 @@ cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_
                             cudaStream_t stream) {
   const int mode = patch_coder_mode();  // the setting covers the rows of matrices as well
   if (mode == 1 || n <= 256 || n > 8192 || (mode == 0 && rows < kHistMinRows))
-    return launch_rows_sort(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, nullptr, 0);
+    return launch_rows_sort(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, 0);
   // The histogram-pruned search first; the sorting kernel then takes the rows it marked.
-  uint32_t call_id = 0;
-  unsigned int *flag1 = nullptr, *flag2 = nullptr;
-  cudaError_t e = chain_flags(&call_id, &flag1, &flag2);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
   const int min_density = 0;  // rows of any density: on matrices this large the search beats the sort on sparse rows too
-  if (n < 1024) e = launch_rows_hist<2>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density, flag1, call_id);
-  else if (n < 4096) e = launch_rows_hist<4>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density, flag1, call_id);
-  else e = launch_rows_hist<8>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density, flag1, call_id);
+  if (n < 1024) e = launch_rows_hist<2>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density);
+  else if (n < 4096) e = launch_rows_hist<4>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density);
+  else e = launch_rows_hist<8>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, min_density);
   if (e != cudaSuccess) return e;
-  return launch_rows_sort(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, flag1, call_id);
+  return launch_rows_sort(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask, flags, stream, 1);
 }
 
 }  // namespace dab

@@ -79,6 +79,15 @@ struct GemmArgs {
   int64_t ldp;
 };
 
+// Number of SMs of the current device (read once per device).
+int sm_count();
+// Opts `kernel` in to `bytes` of dynamic shared memory on the current device unless an earlier call already did.
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes) {
+  return ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), bytes);
+}
+
 cudaError_t launch_binarize(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K,
                             float* alpha, float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags,
                             cudaStream_t stream);
@@ -100,8 +109,6 @@ cudaError_t launch_binarize_patches_pixhist(const dab_conv_desc& d, int32_t Ho, 
 // 3 pixel-histogram coder wherever it applies.
 int patch_coder_mode();
 void set_patch_coder_mode(int mode);
-// Two flag words for a chain of kernels of one call (see PatchArgs in patches.cu) and the call's id.
-cudaError_t chain_flags(uint32_t* call_id, unsigned int** first, unsigned int** second);
 constexpr int32_t kRowMark = -1;  // K of a row or of a tile's first patch that the next kernel of a chain has to code
 cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K, float* alpha,
                              float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags, cudaStream_t stream);
@@ -121,6 +128,5 @@ cudaError_t launch_train_forward(const float* W, int64_t rows, int32_t n, int64_
 cudaError_t launch_train_backward(const float* Wc, int64_t ld_Wc, const uint32_t* mask, int32_t ld_mask,
                                   const int32_t* K, int64_t rows, int32_t n, const float* gWt, int64_t ld_g, float* gW,
                                   int64_t ld_gw, cudaStream_t stream);
-cudaError_t launch_popc_probe(uint32_t* sink, int32_t blocks, int32_t iters, cudaStream_t stream);
 
 }  // namespace dab

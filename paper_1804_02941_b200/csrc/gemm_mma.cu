@@ -229,17 +229,9 @@ inline size_t dynamic_bytes(int kq, int ncap) {
 
 template <int THREADS, int KQ, int MIN_CTAS, int NT_MAX, bool kLanesAreActivations>
 cudaError_t launch_shape(const GemmArgs& args, dim3 grid, int tile_cols, int ncap, cudaStream_t stream) {
-  static bool configured[64] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   auto kernel = binary_gemm_mma_kernel<THREADS, KQ, MIN_CTAS, NT_MAX, kLanesAreActivations>;
-  if (!configured[dev]) {
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynamic_bytes(KQ, NT_MAX));
-    if (e != cudaSuccess) return e;
-    configured[dev] = true;
-  }
+  cudaError_t e = ensure_dynamic_smem(kernel, dynamic_bytes(KQ, NT_MAX));
+  if (e != cudaSuccess) return e;
   kernel<<<grid, THREADS, dynamic_bytes(KQ, ncap), stream>>>(args, tile_cols);
   return cudaGetLastError();
 }
@@ -250,7 +242,7 @@ cudaError_t launch_side(const GemmArgs& args, cudaStream_t stream) {
   // Column tile: the full 256 columns of an accumulator unless that leaves most SMs without a CTA.
   const int64_t gx = (lane_rows + MMA_M - 1) / MMA_M;
   int tile_cols = MMA_NMAX;
-  while (tile_cols > 64 && gx * ((col_rows + tile_cols - 1) / tile_cols) < 2 * 148) tile_cols >>= 1;
+  while (tile_cols > 64 && gx * ((col_rows + tile_cols - 1) / tile_cols) < 2 * sm_count()) tile_cols >>= 1;
   const int64_t gy = (col_rows + tile_cols - 1) / tile_cols;
   if (gx > 0x7FFFFFFF || gy > 65535) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)gx, (unsigned)gy);

@@ -96,7 +96,7 @@ cudaError_t launch_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld
                         int32_t ld_mask, int32_t* K, cudaStream_t stream) {
   const int threads = 256, wpb = threads / 32;
   int64_t blocks = (rows + wpb - 1) / wpb;
-  if (blocks > 148 * 64) blocks = 148 * 64;
+  if (blocks > sm_count() * 64) blocks = sm_count() * 64;
   bool aligned = (reinterpret_cast<uintptr_t>(bits) % 16 == 0) && (ld_bits % 16 == 0);
   if (aligned) {
     const uint32_t magic = (uint32_t)(0x100000000ull / (uint64_t)ld_mask);  // ld_mask >= 4
@@ -104,13 +104,13 @@ cudaError_t launch_pack(const uint8_t* bits, int64_t rows, int32_t n, int64_t ld
     for (int64_t r0 = 0; r0 < rows; r0 += rows_per_launch) {
       const int64_t nr = rows - r0 < rows_per_launch ? rows - r0 : rows_per_launch;
       int64_t pb = (nr * ld_mask + threads - 1) / threads;
-      if (pb > 148 * 32) pb = 148 * 32;
+      if (pb > sm_count() * 32) pb = sm_count() * 32;
       pack_aligned_kernel<<<(unsigned)pb, threads, 0, stream>>>(bits, nr, n, ld_bits, mask, ld_mask, magic, r0);
     }
     if (K) {
       if (ld_mask <= 64) {
         int64_t cb = (rows + threads - 1) / threads;
-        if (cb > 148 * 32) cb = 148 * 32;
+        if (cb > sm_count() * 32) cb = sm_count() * 32;
         count_ones_thread_kernel<<<(unsigned)cb, threads, 0, stream>>>(mask, rows, ld_mask, K);
       } else {
         count_ones_warp_kernel<<<(unsigned)blocks, threads, 0, stream>>>(mask, rows, ld_mask, K);

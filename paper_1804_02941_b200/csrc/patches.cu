@@ -22,13 +22,8 @@ struct PatchArgs {
   int32_t scratch_words;
   int32_t defer_dense;     // leave tiles that look dense to the next kernel of the chain (marks them in pK)
   int32_t dense_num, dense_den;  // a tile is dense if non-zero staged values * dense_den > staged values * dense_num
-  int32_t marked_only;     // code only the tiles marked by the kernel before
-  // Chains of kernels on one stream hand tiles on through marks.  So that a kernel with nothing to do ends at
-  // once, the kernel that marks a tile also writes the call's id to *flag_out, and a marked-only kernel leaves
-  // at entry unless *flag_in holds that id.  (Either pointer may be null: no flag written / always run.)
-  uint32_t call_id;
-  unsigned int* flag_in;
-  unsigned int* flag_out;
+  int32_t marked_only;     // code only the tiles marked by the kernel before (chains of kernels on one stream hand
+                           // tiles on through marks; a CTA none of whose tiles is marked leaves at entry)
   int32_t tile_shape;      // index into kTileShapes forced by the caller, -1: choose
   uint32_t magic_per_ch, magic_in_w;  // ceil(2^32 / d) for d = in_h*in_w and in_w: floor(i/d) = umulhi(i, magic); 0 if d == 1
   const float* x;
@@ -100,16 +95,17 @@ __device__ __forceinline__ int64_t staged_inside(const PatchArgs& a, const TileC
   return (int64_t)a.d.C * max(rows, 0) * max(cols, 0);
 }
 
-// Whether a marked-only kernel has anything to do in this CTA: the call's flag says that some tile was marked at
-// all, then the marks of the CTA's own tiles are read.  Every thread of the CTA gets the same answer.
+// Whether a marked-only kernel has anything to do in this CTA: the marks of the CTA's own tiles are read, one tile
+// per thread at a time.  Every thread of the CTA gets the same answer.
 __device__ __forceinline__ bool has_marked_tile(const PatchArgs& a) {
-  if (a.flag_in && *reinterpret_cast<volatile unsigned int*>(a.flag_in) != a.call_id) return false;
   const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
-  for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+  int any = 0;
+  for (int64_t tile_id = blockIdx.x + (int64_t)threadIdx.x * gridDim.x; tile_id < total_tiles;
+       tile_id += (int64_t)blockDim.x * gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
-    if (a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] == kDenseMark) return true;
+    any |= a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] == kDenseMark;
   }
-  return false;
+  return __syncthreads_or(any) != 0;
 }
 
 #ifndef DAB_WARP_MINBLOCKS
@@ -150,10 +146,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
       __syncthreads();
       const int64_t staged = staged_inside(a, t);
       if ((int64_t)tile_nonzero * a.dense_den > a.dense_num * staged) {
-        if (threadIdx.x == 0) {
-          a.pK[first_patch] = kDenseMark;
-          if (a.flag_out) *a.flag_out = a.call_id;
-        }
+        if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
         continue;
       }
     } else {
@@ -218,10 +211,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
       __syncthreads();
       const int64_t staged = staged_inside(a, t);
       if ((int64_t)tile_nonzero * a.dense_den > a.dense_num * staged) {
-        if (threadIdx.x == 0) {
-          a.pK[first_patch] = kDenseMark;
-          if (a.flag_out) *a.flag_out = a.call_id;
-        }
+        if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
         continue;
       }
     }
@@ -332,10 +322,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
     const uint32_t tkmin = ht.kmin, tkmax = ht.kmax;
     const bool any_nonzero = tkmin <= tkmax;
     if (any_nonzero && key_range_nonfinite(tkmin, tkmax)) {
-      if (threadIdx.x == 0) {
-        a.pK[first_patch] = kDenseMark;
-        if (a.flag_out) *a.flag_out = a.call_id;
-      }
+      if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
       continue;
     }
     const float lo = any_nonzero ? key_value(tkmin) : 0.0f, hi = any_nonzero ? key_value(tkmax) : 0.0f;
@@ -392,10 +379,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
       for (int w = rounds + lane; w < a.ldp; w += 32) mrow[w] = 0u;
     }
     __syncthreads();
-    if (threadIdx.x == 0 && ht.retry) {
-      a.pK[first_patch] = kDenseMark;
-      if (a.flag_out) *a.flag_out = a.call_id;
-    }
+    if (threadIdx.x == 0 && ht.retry) a.pK[first_patch] = kDenseMark;
   }
 }
 
@@ -485,40 +469,17 @@ __global__ void __launch_bounds__(256) sign_rows_kernel(const float* __restrict_
 cudaError_t launch_sign_rows(const float* values, int64_t rows, int32_t n, int64_t ld_values, int32_t* K, float* alpha,
                              float* beta, uint32_t* mask, int32_t ld_mask, uint32_t* flags, cudaStream_t stream) {
   int64_t blocks = (rows + 7) / 8;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   sign_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(values, rows, n, ld_values, K, alpha, beta, mask, ld_mask,
                                                         flags);
   return cudaGetLastError();
 }
 
 // 0: by tile density (default), 1: sort-based coders only, 2: histogram-pruned coder wherever it applies.
-static int g_patch_coder_mode = 0;
+static std::atomic<int> g_patch_coder_mode{0};
 
-// Flags of the kernel chains (see PatchArgs): two words per call, taken in turn from a small ring.
-constexpr int kChainSlots = 256;
-static __device__ unsigned int g_chain_flags[2 * kChainSlots];
-static std::atomic<uint32_t> g_chain_calls{0};
-
-cudaError_t chain_flags(uint32_t* call_id, unsigned int** first, unsigned int** second) {
-  static unsigned int* base[64] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!base[dev]) {
-    void* ptr = nullptr;
-    if ((e = cudaGetSymbolAddress(&ptr, g_chain_flags)) != cudaSuccess) return e;
-    base[dev] = static_cast<unsigned int*>(ptr);
-  }
-  uint32_t id = ++g_chain_calls;
-  if (id == 0) id = ++g_chain_calls;  // 0 is what the flags hold before any call
-  *call_id = id;
-  *first = base[dev] + 2 * (id % kChainSlots);
-  *second = *first + 1;
-  return cudaSuccess;
-}
-int patch_coder_mode() { return g_patch_coder_mode; }
-void set_patch_coder_mode(int mode) { g_patch_coder_mode = mode; }
+int patch_coder_mode() { return g_patch_coder_mode.load(std::memory_order_relaxed); }
+void set_patch_coder_mode(int mode) { g_patch_coder_mode.store(mode, std::memory_order_relaxed); }
 
 // Tile shapes tried, largest first.
 static const int kTileShapes[][2] = {{8, 8}, {4, 8}, {4, 4}, {2, 4}, {2, 2}, {1, 2}, {1, 1}};
@@ -547,7 +508,7 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
   // tile loads overlap other CTAs' sorting), 16 for larger groups (fewer, larger tiles matter more)
   const int want_warps = groups >= 4 ? 24 : 16;
   const int want_ctas = (want_warps * 32 + threads - 1) / threads;
-  const int64_t want_tiles = 2 * 148;
+  const int64_t want_tiles = 2 * sm_count();
   int best = -1, best_ctas = 0, small = -1;
   size_t best_smem = 0, small_smem = 0;
   bool settled = false;
@@ -574,10 +535,10 @@ static cudaError_t launch_patches(Kernel kern, PatchArgs& a, size_t fixed_bytes,
   a.tile_shape = best;
   set_tile(a.d, a.Ho, a.Wo, kTileShapes[best], &a);
   if (shape_only) return cudaSuccess;  // the caller wanted the tile this kernel would take
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)best_smem);
+  cudaError_t e = ensure_dynamic_smem(kern, best_smem);
   if (e != cudaSuccess) return e;
   int64_t tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
-  int64_t blocks = tiles < 148 * 8 ? tiles : 148 * 8;
+  int64_t blocks = tiles < sm_count() * 8 ? tiles : sm_count() * 8;
   kern<<<(unsigned)blocks, threads, best_smem, stream>>>(a);
   return cudaGetLastError();
 }
@@ -651,7 +612,6 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   a.defer_dense = 0; a.marked_only = 0; a.tile_shape = -1;
   a.x = x; a.pK = pK; a.pgamma = pgamma; a.pdelta = pdelta; a.pflags = pflags; a.pmask = pmask; a.ldp = ldp;
   a.dense_num = 1; a.dense_den = 0;  // no tile counts as dense unless a chain below says so
-  a.call_id = 0; a.flag_in = nullptr; a.flag_out = nullptr;
   if (a.n <= 256) return launch_patches_warp<8, false>(a, stream);
   const int mode = patch_coder_mode();
   cudaError_t e;
@@ -679,18 +639,15 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
     }
     return launch_group_for(a, stream, false);
   }
-  unsigned int *flag1 = nullptr, *flag2 = nullptr;
-  if ((e = chain_flags(&a.call_id, &flag1, &flag2)) != cudaSuccess) return e;
   // The histogram-pruned coder runs on the tile shape of the group kernel, which ends every chain by taking the
   // tiles nobody else settled.  Its 16-bit offsets must reach the whole (odd-pitched) tile.
   if ((e = launch_group_for(a, stream, /*shape_only=*/true)) != cudaSuccess) return e;
   const bool hist_fits = (size_t)a.d.C * ((a.in_h * a.pitch) | 1) <= 65535;
   if (mode == 2) {  // everything through the histogram coder
     if (hist_fits) {
-      a.flag_out = flag2;
       e = launch_hist_for(a, stream);
       if (e != cudaSuccess) return e;
-      a.marked_only = 1; a.flag_in = flag2; a.flag_out = nullptr;
+      a.marked_only = 1;
     }
     return launch_group_for(a, stream, false);
   }
@@ -702,7 +659,7 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
     a.tile_shape = -1;
     return launch_group_for(a, stream, false);
   }
-  a.defer_dense = 1; a.flag_out = flag1;
+  a.defer_dense = 1;
   if (a.n <= 576) {
     a.dense_num = 256; a.dense_den = a.n;  // expected non-zeros per patch above the 256 one warp sorts with 8 keys per lane
     a.tile_shape = -1;  // the one-warp kernel picks its own tile; the two kernels after it take it over
@@ -712,12 +669,10 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
     e = launch_group_for(a, stream, false);
   }
   if (e != cudaSuccess) return e;
-  a.defer_dense = 0; a.marked_only = 1; a.flag_in = flag1; a.flag_out = nullptr;
+  a.defer_dense = 0; a.marked_only = 1;
   if ((size_t)a.d.C * ((a.in_h * a.pitch) | 1) <= 65535) {  // (the first kernel may have taken another tile)
-    a.flag_out = flag2;
     e = launch_hist_for(a, stream);
     if (e != cudaSuccess) return e;
-    a.flag_in = flag2; a.flag_out = nullptr;
   }
   return launch_group_for(a, stream, false);
 }

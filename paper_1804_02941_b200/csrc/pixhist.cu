@@ -652,6 +652,7 @@ bool choose_pix_tile(PixArgs* a, size_t budget, int ctas_per_sm, size_t* smem_ou
   int best_th = 0, best_tw = 0;
   size_t best_smem = 0;
   const double per_patch = 5000.0 + 5.0 * a->n;
+  const int sms = sm_count();
   for (int th = 8; th >= 1; --th) {
     for (int tw = 8; tw >= 1; --tw) {
       if ((th > a->Ho && th > 1) || (tw > a->Wo && tw > 1)) continue;
@@ -661,7 +662,7 @@ bool choose_pix_tile(PixArgs* a, size_t budget, int ctas_per_sm, size_t* smem_ou
       const size_t smem = pix_smem_bytes<WARPS, BPL, KHW, ListT, kTable>(t);
       if (smem > budget) continue;
       const int64_t tiles = (int64_t)t.tiles_h * t.tiles_w * t.d.N;
-      const int64_t slots = (int64_t)148 * ctas_per_sm;
+      const int64_t slots = (int64_t)sms * ctas_per_sm;
       const double waves = (double)((tiles + slots - 1) / slots);
       const int rounds = (t.TH * t.TW + WARPS - 1) / WARPS;
       const double cost = waves * (4.6 * t.pix * t.d.C + rounds * per_patch) * sqrt((double)ctas_per_sm);  // resident CTAs share the issue slots
@@ -680,10 +681,10 @@ constexpr size_t kSmemPerSm = 228 * 1024, kSmemCtaReserve = 1024, kSmemCtaMax = 
 template <int WARPS, int MINB, int BPL, int KHW, typename ListT, bool kTable>
 cudaError_t launch_pix_minb(PixArgs& a, size_t smem, cudaStream_t stream) {
   auto kern = binarize_patches_pixhist_kernel<WARPS, MINB, BPL, KHW, ListT, kTable>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   const int64_t tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
-  const int64_t blocks = tiles < 148 * MINB ? tiles : 148 * MINB;
+  const int64_t blocks = tiles < sm_count() * MINB ? tiles : sm_count() * MINB;
   kern<<<(unsigned)blocks, WARPS * 32, smem, stream>>>(a);
   return cudaGetLastError();
 }
@@ -733,11 +734,11 @@ cudaError_t launch_fixup(const PixArgs& a, cudaStream_t stream) {
   const int sw = scratch_words_for(a.n, kFixWarps);
   const size_t smem = sizeof(GroupShared) + sizeof(uint32_t) * (size_t)sw + sizeof(int) * kFixThreads;
   auto kern = binarize_patches_fixup_kernel<R>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   const int64_t total = (int64_t)a.d.N * a.Ho * a.Wo;
   int64_t blocks = (total + kFixThreads - 1) / kFixThreads;
-  if (blocks > 148 * 4) blocks = 148 * 4;
+  if (blocks > sm_count() * 4) blocks = sm_count() * 4;
   kern<<<(unsigned)blocks, kFixThreads, smem, stream>>>(a, sw);
   return cudaGetLastError();
 }

@@ -35,10 +35,11 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 
-// Bounded wait for the phase with the given parity.  Returns false after kWaitCycles and counts the failure
+// Bounded wait for the phase with the given parity.  Returns false after `limit` cycles and counts the failure
 // in *failures (device global); the caller then stops waiting on anything (dead stays set) but keeps its
 // control flow, so that every thread still reaches every barrier and the CTA ends.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, bool& dead, unsigned int* failures) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, bool& dead, unsigned int* failures,
+                                          long long limit = kWaitCycles) {
   if (dead) return false;
   const long long t0 = clock64();
   for (;;) {
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, bool& d
         : "r"(bar), "r"(parity)
         : "memory");
     if (done) return true;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       dead = true;
       atomicAdd(failures, 1u);
       return false;

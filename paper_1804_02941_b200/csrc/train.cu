@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) train_backward_kernel(const float* __rest
 
 unsigned grid_for_rows(int64_t rows) {
   int64_t blocks = (rows + 7) / 8;
-  return (unsigned)(blocks > 148 * 16 ? 148 * 16 : (blocks < 1 ? 1 : blocks));
+  return (unsigned)(blocks > sm_count() * 16 ? sm_count() * 16 : (blocks < 1 ? 1 : blocks));
 }
 
 }  // namespace

@@ -414,7 +414,7 @@ cudaError_t launch_wbin_conv(const dab_conv_desc& d, int32_t Ho, int32_t Wo, con
   wbin_pixmax_kernel<<<(unsigned)((pixels + 255) / 256), 256, 0, stream>>>(x, pixmax, d.C, HW, pixels);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(wbin_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  e = ensure_dynamic_smem(wbin_conv_kernel, smem);
   if (e != cudaSuccess) return e;
   wbin_conv_kernel<<<dim3((unsigned)gx, (unsigned)gy), WB_THREADS, smem, stream>>>(a);
   return cudaGetLastError();

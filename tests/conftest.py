@@ -24,3 +24,19 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def output_guards(request):
+    """GPU tests: every output tensor the binding creates sits between guard zones, verified after the test (the
+    stand-in for a memory checker: a kernel that writes just outside an output fails the test that ran it)."""
+    if "gpu" not in request.keywords:
+        yield
+        return
+    import paper_1804_02941_b200 as d
+    d.guards_enable(True)
+    try:
+        yield
+        d.guards_check()
+    finally:
+        d.guards_enable(False)
