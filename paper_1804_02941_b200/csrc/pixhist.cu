@@ -22,9 +22,15 @@
 #include "histcode.cuh"
 #include "rowcode.cuh"
 
+#ifndef DAB_PIX_UNROLL
+#define DAB_PIX_UNROLL 4   // channels of one pixel a warp keeps in flight in the per-tile passes
+#endif
+
 namespace dab {
 
 namespace {
+
+constexpr int kPixUnroll = DAB_PIX_UNROLL;
 
 constexpr int kFixWarps = 8;      // warps of the kernel that sorts the marked patches
 constexpr int kFixThreads = kFixWarps * 32;
@@ -215,7 +221,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
         if (o >= 0) {
           const float* src = ximg + o;
           const unsigned saddr = (unsigned)__cvta_generic_to_shared(tile + p);
-#pragma unroll 4
+#pragma unroll kPixUnroll
           for (int c = warp; c < C; c += WARPS)
             asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(saddr + 4u * (unsigned)(c * chw)),
                          "l"(src + (int64_t)c * plane) : "memory");
@@ -229,7 +235,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     {  // range of the non-zero values (-0.0 counts as zero everywhere below: every use is a comparison)
       uint32_t kmin = kPadKey, kmax = 0u;
       for (int p = lane; p < pixn; p += 32) {
-#pragma unroll 4
+#pragma unroll kPixUnroll
         for (int c = warp; c < C; c += WARPS) {
           const float v = tile[c * chw + p];
           const uint32_t key = order_key(v);
@@ -256,7 +262,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     }
     // ---- per pixel: count and fp64 sum per bucket ----
     for (int p = lane; p < pixn; p += 32) {
-#pragma unroll 4
+#pragma unroll kPixUnroll
       for (int c = warp; c < C; c += WARPS) {
         const float v = tile[c * chw + p];
         if (v != 0.0f) {
@@ -284,7 +290,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     __syncthreads();
     // ---- per pixel: channel indices ordered by bucket; the cursors end as inclusive cumulative counts ----
     for (int p = lane; p < pixn; p += 32) {
-#pragma unroll 4
+#pragma unroll kPixUnroll
       for (int c = warp; c < C; c += WARPS) {
         const float v = tile[c * chw + p];
         if (v != 0.0f) {
@@ -692,29 +698,37 @@ cudaError_t launch_pix_minb(PixArgs& a, size_t smem, cudaStream_t stream) {
 #ifndef DAB_PIX_WARPS
 #define DAB_PIX_WARPS 8
 #endif
+#ifndef DAB_PIX_FOUR_CTAS_UPTO_BPL
+#define DAB_PIX_FOUR_CTAS_UPTO_BPL 2   // buckets per lane up to which four CTAs per SM (64 registers a thread) are tried
+#endif
 
-// Three, two or one CTA per SM: the most resident CTAs whose best tile costs no more than 1.25 x the best of all.
+// Four (short rows only), three, two or one CTA per SM: the most resident CTAs whose best tile costs no more than
+// 1.25 x the best of all.
 template <int BPL, int KHW, typename ListT, bool kTable>
 cudaError_t launch_pix(PixArgs& a, cudaStream_t stream, bool* applicable) {
   constexpr int W = DAB_PIX_WARPS;
-  PixArgs cand[3] = {a, a, a};
-  size_t smem[3] = {0, 0, 0};
-  double cost[3] = {0, 0, 0};
-  bool ok[3];
+  constexpr int kMostCtas = BPL <= DAB_PIX_FOUR_CTAS_UPTO_BPL ? 4 : 3;
+  PixArgs cand[4] = {a, a, a, a};
+  size_t smem[4] = {0, 0, 0, 0};
+  double cost[4] = {0, 0, 0, 0};
+  bool ok[4] = {false, false, false, false};
   double best = 0.0;
-  for (int i = 0; i < 3; ++i) {
-    const int ctas = 3 - i;
+  for (int ctas = kMostCtas; ctas >= 1; --ctas) {
     size_t budget = kSmemPerSm / ctas - kSmemCtaReserve;
     if (budget > kSmemCtaMax) budget = kSmemCtaMax;
+    const int i = ctas - 1;
     ok[i] = choose_pix_tile<W, BPL, KHW, ListT, kTable>(&cand[i], budget, ctas, &smem[i], &cost[i]);
     if (ok[i] && (best == 0.0 || cost[i] < best)) best = cost[i];
   }
-  *applicable = ok[0] || ok[1] || ok[2];
+  *applicable = ok[0] || ok[1] || ok[2] || ok[3];
   if (!*applicable) return cudaSuccess;
-  if (ok[0] && cost[0] <= 1.25 * best) { a = cand[0]; return launch_pix_minb<W, 3, BPL, KHW, ListT, kTable>(a, smem[0], stream); }
+  if constexpr (kMostCtas == 4) {
+    if (ok[3] && cost[3] <= 1.25 * best) { a = cand[3]; return launch_pix_minb<W, 4, BPL, KHW, ListT, kTable>(a, smem[3], stream); }
+  }
+  if (ok[2] && cost[2] <= 1.25 * best) { a = cand[2]; return launch_pix_minb<W, 3, BPL, KHW, ListT, kTable>(a, smem[2], stream); }
   if (ok[1] && cost[1] <= 1.25 * best) { a = cand[1]; return launch_pix_minb<W, 2, BPL, KHW, ListT, kTable>(a, smem[1], stream); }
-  a = cand[2];
-  return launch_pix_minb<W, 1, BPL, KHW, ListT, kTable>(a, smem[2], stream);
+  a = cand[0];
+  return launch_pix_minb<W, 1, BPL, KHW, ListT, kTable>(a, smem[0], stream);
 }
 
 // Reciprocal table for rows of fewer than 2048 values; 8-bit channel indices where the channel count allows (3 x 3

@@ -440,6 +440,22 @@ __device__ __forceinline__ RowResult group_select(const uint32_t (&r)[E], int m,
     }
   }
   RowResult res;
+  if (W == 1) {
+    // every lane holds the winner: the two means are formed side by side in lanes 0 and 1 (the same two divisions as
+    // finish_row, one after the other's latency instead of behind it)
+    const double num = lane == 1 ? __dsub_rn(T, bP) : bP;
+    const double den = lane == 1 ? (double)(n - bS) : (double)bS;
+    const double mean = __ddiv_rn(num, den);
+    const double m_lo = __shfl_sync(0xFFFFFFFFu, mean, 0), m_hi = __shfl_sync(0xFFFFFFFFu, mean, 1);
+    const bool low_side = fabs(m_lo) > fabs(m_hi);
+    res.K = low_side ? bS : n - bS;
+    res.alpha = (float)(low_side ? m_lo : m_hi);
+    res.beta = (float)(low_side ? m_hi : m_lo);
+    res.flags = 0u;
+    res.tkey = bT;
+    res.mode = low_side ? 1 : 0;
+    return res;
+  }
   if (tig == 0) res = finish_row(bP, bS, bT, T, n);
   return res;
 }
