@@ -230,3 +230,92 @@ def im2col(x, kh, kw, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     out = np.zeros((N * Ho * Wo, Cc * kh * kw), np.float32)
     lib().oracle_im2col(C.byref(d), _p(x), _p(out))
     return out
+
+
+# ------------------------------------------------------------------------------------------------------------
+# Whole networks: the full-precision layers around the binarized ones, and the chain
+# ------------------------------------------------------------------------------------------------------------
+def conv_dense(x, w, kh, kw, stride=(1, 1), pad=(0, 0), bias=None) -> np.ndarray:
+    """x (*) W (+ bias) with full-precision filters W [Cout x C*kh*kw]; fp64 sums in (c, kh, kw) order, fp32 out."""
+    x = np.ascontiguousarray(x, np.float32)
+    w = np.ascontiguousarray(w, np.float32)
+    N, Cc, H, W = x.shape
+    Cout, n = w.shape
+    assert n == Cc * kh * kw
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    d = _desc(x.shape, Cout, kh, kw, stride, pad)
+    y = np.zeros((N, Cout, Ho, Wo), np.float32)
+    b = None if bias is None else np.ascontiguousarray(bias, np.float32)
+    lib().oracle_conv_dense(C.byref(d), _p(x), _p(w), _p(b), _p(y))
+    return y
+
+
+def affine(x, scale, shift) -> np.ndarray:
+    x = np.ascontiguousarray(x, np.float32)
+    N, Cc = x.shape[0], x.shape[1]
+    hw = int(np.prod(x.shape[2:]))
+    y = np.zeros_like(x)
+    lib().oracle_affine(_p(x), C.c_int64(N), C.c_int32(Cc), C.c_int64(hw), _p(np.ascontiguousarray(scale, np.float32)),
+                        _p(np.ascontiguousarray(shift, np.float32)), _p(y))
+    return y
+
+
+def relu(x) -> np.ndarray:
+    x = np.ascontiguousarray(x, np.float32)
+    y = np.zeros_like(x)
+    lib().oracle_relu(_p(x), C.c_int64(x.size), _p(y))
+    return y
+
+
+def maxpool(x, kh, kw, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
+    x = np.ascontiguousarray(x, np.float32)
+    N, Cc, H, W = x.shape
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    d = _desc(x.shape, Cc, kh, kw, stride, pad)
+    y = np.zeros((N, Cc, Ho, Wo), np.float32)
+    lib().oracle_maxpool(C.byref(d), _p(x), _p(y))
+    return y
+
+
+def add(a, b) -> np.ndarray:
+    a = np.ascontiguousarray(a, np.float32)
+    b = np.ascontiguousarray(b, np.float32)
+    assert a.shape == b.shape
+    y = np.zeros_like(a)
+    lib().oracle_add(_p(a), _p(b), C.c_int64(a.size), _p(y))
+    return y
+
+
+def network_layer(layer, x, saved):
+    """One layer of a chain (a dict from dab_synth.networks): returns (output, saved).  `saved` is the tensor a
+    shortcut holds; layers with on_saved = True transform it instead of the running tensor."""
+    kind = layer["kind"]
+    src = saved if layer.get("on_saved") else x
+    if kind == "conv_dense":
+        out = conv_dense(src, layer["w"], layer["kh"], layer["kw"], layer["stride"], layer["pad"], layer.get("bias"))
+    elif kind == "conv_binary":
+        wb = binarize(layer["w"])
+        out = conv(src, wb.e, wb.alpha, wb.beta, layer["kh"], layer["kw"], layer["stride"], layer["pad"], details=False).y
+    elif kind == "affine":
+        out = affine(src, layer["scale"], layer["shift"])
+    elif kind == "relu":
+        out = relu(src)
+    elif kind == "maxpool":
+        out = maxpool(src, layer["kh"], layer["kw"], layer["stride"], layer["pad"])
+    elif kind == "save":
+        return x, x.copy()
+    elif kind == "add":
+        return add(x, saved), saved
+    else:
+        raise ValueError(kind)
+    return (x, out) if layer.get("on_saved") else (out, saved)
+
+
+def network_forward(layers, x, keep=False):
+    """The whole chain on the CPU.  keep: also return the running tensor after every layer."""
+    saved, outs = None, []
+    for layer in layers:
+        x, saved = network_layer(layer, x, saved)
+        if keep:
+            outs.append(x)
+    return (x, outs) if keep else x

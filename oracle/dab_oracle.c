@@ -380,3 +380,79 @@ void oracle_theorem4(const float* W, const uint8_t* e, const int32_t* K, int64_t
     }
   }
 }
+
+/* ------------------------------------------------------------------------------------------------------------
+ * Full-precision layers around the binarized ones (Section 5.1), plain definitions.
+ * ------------------------------------------------------------------------------------------------------------ */
+void oracle_conv_dense(const oracle_conv_desc* d, const float* x, const float* w, const float* bias, float* y) {
+  int32_t Ho, Wo;
+  int64_t outputs, oi;
+  int32_t n = d->C * d->kh * d->kw;
+  conv_out_size(d, &Ho, &Wo);
+  outputs = (int64_t)d->N * d->Cout * Ho * Wo;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static) num_threads(g_threads)
+#endif
+  for (oi = 0; oi < outputs; ++oi) {
+    int32_t wo = (int32_t)(oi % Wo);
+    int32_t ho = (int32_t)((oi / Wo) % Ho);
+    int32_t co = (int32_t)((oi / ((int64_t)Wo * Ho)) % d->Cout);
+    int32_t img = (int32_t)(oi / ((int64_t)Wo * Ho * d->Cout));
+    double acc = 0.0;
+    int32_t c, r, s;
+    for (c = 0; c < d->C; ++c)
+      for (r = 0; r < d->kh; ++r)
+        for (s = 0; s < d->kw; ++s) {
+          int32_t h = ho * d->stride_h - d->pad_h + r, wq = wo * d->stride_w - d->pad_w + s;
+          double xv = 0.0, prod;
+          if (h >= 0 && h < d->H && wq >= 0 && wq < d->W) xv = (double)x[(((int64_t)img * d->C + c) * d->H + h) * d->W + wq];
+          prod = xv * (double)w[(int64_t)co * n + ((int64_t)c * d->kh + r) * d->kw + s];
+          acc = acc + prod;
+        }
+    if (bias) acc = acc + (double)bias[co];
+    y[oi] = (float)acc;
+  }
+}
+
+void oracle_affine(const float* x, int64_t N, int32_t C, int64_t HW, const float* scale, const float* shift, float* y) {
+  int64_t total = N * C * HW, i;
+  for (i = 0; i < total; ++i) {
+    int32_t c = (int32_t)((i / HW) % C);
+    double t = (double)scale[c] * (double)x[i];
+    y[i] = (float)(t + (double)shift[c]);
+  }
+}
+
+void oracle_relu(const float* x, int64_t count, float* y) {
+  int64_t i;
+  for (i = 0; i < count; ++i) y[i] = x[i] > 0.0f ? x[i] : 0.0f;
+}
+
+void oracle_maxpool(const oracle_conv_desc* d, const float* x, float* y) {
+  int32_t Ho, Wo;
+  int64_t outputs, oi;
+  conv_out_size(d, &Ho, &Wo);
+  outputs = (int64_t)d->N * d->C * Ho * Wo;
+  for (oi = 0; oi < outputs; ++oi) {
+    int32_t wo = (int32_t)(oi % Wo);
+    int32_t ho = (int32_t)((oi / Wo) % Ho);
+    int64_t plane = oi / ((int64_t)Wo * Ho);
+    int32_t r, s, seen = 0;
+    float best = 0.0f;
+    for (r = 0; r < d->kh; ++r)
+      for (s = 0; s < d->kw; ++s) {
+        int32_t h = ho * d->stride_h - d->pad_h + r, wq = wo * d->stride_w - d->pad_w + s;
+        if (h >= 0 && h < d->H && wq >= 0 && wq < d->W) {
+          float v = x[(plane * d->H + h) * d->W + wq];
+          if (!seen || v > best) best = v;
+          seen = 1;
+        }
+      }
+    y[oi] = best;
+  }
+}
+
+void oracle_add(const float* a, const float* b, int64_t count, float* y) {
+  int64_t i;
+  for (i = 0; i < count; ++i) y[i] = a[i] + b[i];
+}

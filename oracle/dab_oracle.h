@@ -130,6 +130,25 @@ void oracle_theorem4(const float* W, const uint8_t* e, const int32_t* K, int64_t
 /* Patch extraction alone (explicit loops), rows = N*Ho*Wo, row length C*kh*kw. */
 void oracle_im2col(const oracle_conv_desc* d, const float* x, float* patches);
 
+/*
+ * The layers around the binarized ones when whole networks are chained (Section 5.1: the first layer, and the last
+ * one in Sketch-A-Net, stay full precision; Appendix "Experimental details" for the glue).  The paper gives no
+ * arithmetic for them; each is written here as its plain definition, fp64 inside, one rounding to fp32.
+ *
+ * oracle_conv_dense  y = x (*) W (+ bias): for every output the products are summed in fp64 in element order
+ *                    (c, kh, kw), each product and sum rounded on its own, zero padding; W is [Cout][C*kh*kw].
+ * oracle_affine      y = scale[c] * x + shift[c] per channel (a folded normalisation layer); x is N x C x HW.
+ * oracle_relu        y = x > 0 ? x : 0  (-0.0 and NaN give +0.0).
+ * oracle_maxpool     maximum over the kh x kw window (positions outside the image are skipped); d->C channels,
+ *                    d->Cout ignored; output size as for a convolution of the same geometry.
+ * oracle_add         y = a + b in fp32 (the shortcut of a residual block).
+ */
+void oracle_conv_dense(const oracle_conv_desc* d, const float* x, const float* w, const float* bias, float* y);
+void oracle_affine(const float* x, int64_t N, int32_t C, int64_t HW, const float* scale, const float* shift, float* y);
+void oracle_relu(const float* x, int64_t count, float* y);
+void oracle_maxpool(const oracle_conv_desc* d, const float* x, float* y);
+void oracle_add(const float* a, const float* b, int64_t count, float* y);
+
 #ifdef __cplusplus
 }
 #endif
