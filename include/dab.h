@@ -286,6 +286,61 @@ dab_status dab_binary_conv_static(const dab_conv_desc* desc, const float* d_x, c
                                   void* stream);
 
 /*
+ * Whole networks (Section 5.1: Sketch-A-Net, ResNet-18 and GoogLeNet with "all but the first [and last] layer
+ * binarized"; Appendix "Experimental details": no bias in the binarized layers).  A network is a HOST array of
+ * dab_layer records run one after the other on a running tensor (NCHW fp32); a second, remembered tensor carries
+ * the shortcut of a residual block.  The pointers inside a record are DEVICE pointers owned by the caller.
+ *
+ *   DAB_LAYER_CONV_DENSE   full-precision convolution: d_weights [Cout x C*kh*kw] fp32, d_bias Cout fp32 or NULL;
+ *                          products summed in fp64 in element order (c, kh, kw), one rounding to fp32
+ *   DAB_LAYER_CONV_BINARY  dab_binary_conv with the filters coded by dab_binarize (d_wmask, ldw, d_wK, d_walpha, d_wbeta)
+ *   DAB_LAYER_AFFINE       y = d_scale[c] * x + d_shift[c] per channel, in fp64, one rounding (a folded normalisation)
+ *   DAB_LAYER_RELU         y = x > 0 ? x : 0
+ *   DAB_LAYER_MAXPOOL      maximum over the kh x kw window, positions outside the image skipped
+ *   DAB_LAYER_SAVE         remember (a copy of) the running tensor
+ *   DAB_LAYER_ADD          running tensor + remembered tensor (same shape), fp32
+ * on_saved != 0 (CONV_DENSE, AFFINE, RELU, MAXPOOL): the layer transforms the remembered tensor instead of the
+ * running one (the 1x1 projection of a shortcut).  Fully connected layers are convolutions whose kernel covers
+ * their whole input.  Fields a kind does not use are ignored.
+ *
+ * dab_network_output_shape  shape of the running tensor after the last layer.
+ * dab_network_workspace     bytes of scratch dab_network_forward needs (four tensors of the largest size in the chain
+ *                           plus the scratch of its largest binarized layer); 0 if the chain is invalid.
+ * dab_network_forward       queues every layer on `stream` and returns without synchronising.  d_y receives the
+ *                           running tensor after the last layer.  h_layer_outputs (host array of `count` device
+ *                           pointers, or NULL; entries may be NULL): where given, layer i writes its output there
+ *                           instead of into the workspace, so that a caller can inspect every intermediate tensor.
+ * DAB_ERR_INVALID_ARG for a chain that does not fit together (shapes, missing pointers, ADD without SAVE),
+ * DAB_ERR_UNSUPPORTED for a binarized layer with C*kh*kw > DAB_MAX_N, DAB_ERR_WORKSPACE as elsewhere.
+ */
+typedef enum {
+  DAB_LAYER_CONV_DENSE = 0, DAB_LAYER_CONV_BINARY = 1, DAB_LAYER_AFFINE = 2, DAB_LAYER_RELU = 3, DAB_LAYER_MAXPOOL = 4,
+  DAB_LAYER_SAVE = 5, DAB_LAYER_ADD = 6
+} dab_layer_kind;
+
+typedef struct {
+  int32_t kind;      /* dab_layer_kind */
+  int32_t on_saved;
+  int32_t Cout, kh, kw, stride_h, stride_w, pad_h, pad_w;
+  int32_t ldw;
+  const float* d_weights;
+  const float* d_bias;
+  const uint32_t* d_wmask;
+  const int32_t* d_wK;
+  const float* d_walpha;
+  const float* d_wbeta;
+  const float* d_scale;
+  const float* d_shift;
+} dab_layer;
+
+dab_status dab_network_output_shape(const dab_layer* layers, int32_t count, int32_t N, int32_t C, int32_t H, int32_t W,
+                                    int32_t* Cout, int32_t* Ho, int32_t* Wo);
+size_t dab_network_workspace(const dab_layer* layers, int32_t count, int32_t N, int32_t C, int32_t H, int32_t W);
+dab_status dab_network_forward(const dab_layer* layers, int32_t count, int32_t N, int32_t C, int32_t H, int32_t W,
+                               const float* d_x, float* d_y, void* d_workspace, size_t workspace_bytes,
+                               float* const* h_layer_outputs, void* stream);
+
+/*
  * Which kernel forms the AND-popcounts of dab_binary_gemm and of every convolution entry point (Section 4.2
  * counts set bits with population-count instructions; an AND-popcount over n bits is also the dot product of
  * the two rows written as 0/1 bytes, which the tensor cores form exactly in 32-bit integers):

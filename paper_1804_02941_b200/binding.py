@@ -24,7 +24,8 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_conv_output_size", "dab_binary_conv_workspace", "dab_binary_conv", "dab_binarize_patches",
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
-           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward", "dab_set_patch_coder", "dab_get_patch_coder", "dab_binary_conv_host_async", "dab_binary_conv_host_wait")
+           "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward", "dab_set_patch_coder", "dab_get_patch_coder", "dab_binary_conv_host_async", "dab_binary_conv_host_wait",
+           "dab_network_output_shape", "dab_network_workspace", "dab_network_forward")
 
 
 class DabError(RuntimeError):
@@ -83,6 +84,10 @@ def lib() -> C.CDLL:
         L.dab_get_patch_coder.argtypes = []
         L.dab_get_contraction.argtypes = []
         L.dab_contraction_wait_failures.argtypes = [vp]
+        L.dab_network_output_shape.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.dab_network_workspace.restype = C.c_size_t
+        L.dab_network_workspace.argtypes = [vp, i32, i32, i32, i32, i32]
+        L.dab_network_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, C.c_size_t, vp, vp]
         _lib = L
     return _lib
 
@@ -478,3 +483,81 @@ def dab_contraction_wait_failures() -> int:
     c = C.c_uint32(0)
     _check(lib().dab_contraction_wait_failures(C.byref(c)), "dab_contraction_wait_failures")
     return int(c.value)
+
+
+# ------------------------------------------------------------------------------------------------------------
+# Whole networks (dab_network_forward): the layer records are filled from torch tensors; nothing is computed here
+# ------------------------------------------------------------------------------------------------------------
+LAYER_KINDS = {"conv_dense": 0, "conv_binary": 1, "affine": 2, "relu": 3, "maxpool": 4, "save": 5, "add": 6}
+
+
+class Layer(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("kind", "on_saved", "Cout", "kh", "kw", "stride_h", "stride_w", "pad_h", "pad_w", "ldw")] + \
+               [(k, C.c_void_p) for k in ("d_weights", "d_bias", "d_wmask", "d_wK", "d_walpha", "d_wbeta", "d_scale", "d_shift")]
+
+
+class Network:
+    """A chain of layers resident on a device: the C records plus the tensors they point to (kept alive here).
+    layers: dicts as produced by dab_synth.networks ("kind", geometry, numpy or torch weights); the filters of the
+    binarized layers are coded once, by dab_binarize, when the network is built."""
+
+    def __init__(self, layers, device="cuda"):
+        self.device = torch.device(device)
+        self.keep = []
+        self.records = (Layer * len(layers))()
+        self.kinds = [l["kind"] for l in layers]
+        for rec, l in zip(self.records, layers):
+            rec.kind = LAYER_KINDS[l["kind"]]
+            rec.on_saved = 1 if l.get("on_saved") else 0
+            if "kh" in l:
+                rec.kh, rec.kw = l["kh"], l["kw"]
+                rec.stride_h, rec.stride_w = l["stride"]
+                rec.pad_h, rec.pad_w = l["pad"]
+            if l["kind"] == "conv_dense":
+                w = self._t(l["w"])
+                rec.Cout, rec.d_weights = w.shape[0], w.data_ptr()
+                if l.get("bias") is not None:
+                    rec.d_bias = self._t(l["bias"]).data_ptr()
+            elif l["kind"] == "conv_binary":
+                coded = dab_binarize(self._t(l["w"]))
+                self.keep.append(coded)
+                rec.Cout, rec.ldw = coded.mask.shape[0], coded.ld
+                rec.d_wmask, rec.d_wK = coded.mask.data_ptr(), coded.K.data_ptr()
+                rec.d_walpha, rec.d_wbeta = coded.alpha.data_ptr(), coded.beta.data_ptr()
+            elif l["kind"] == "affine":
+                rec.d_scale, rec.d_shift = self._t(l["scale"]).data_ptr(), self._t(l["shift"]).data_ptr()
+
+    def _t(self, a):
+        t = a if isinstance(a, torch.Tensor) else torch.from_numpy(a)
+        t = t.to(self.device, torch.float32).contiguous()
+        self.keep.append(t)
+        return t
+
+    def __len__(self):
+        return len(self.records)
+
+
+def dab_network_output_shape(net: Network, x_shape):
+    N, Cc, H, W = x_shape
+    co, ho, wo = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    _check(lib().dab_network_output_shape(net.records, len(net), N, Cc, H, W, C.byref(co), C.byref(ho), C.byref(wo)),
+           "dab_network_output_shape")
+    return co.value, ho.value, wo.value
+
+
+def dab_network_forward(net: Network, x: torch.Tensor, keep_layers: bool = False, layer_shapes=None, stream=None):
+    """Runs the chain on x (N x C x H x W fp32, contiguous).  keep_layers: also return every layer's output tensor
+    (layer_shapes: their shapes, one (C, H, W) per layer, as the caller knows them from the network definition)."""
+    _dev(x, torch.float32, "x")
+    N, Cc, H, W = x.shape
+    co, ho, wo = dab_network_output_shape(net, tuple(x.shape))
+    y = _new((N, co, ho, wo), torch.float32, x.device)
+    need = int(lib().dab_network_workspace(net.records, len(net), N, Cc, H, W))
+    ws = _new(need, torch.uint8, x.device)
+    outs, ptrs = None, None
+    if keep_layers:
+        outs = [_new((N,) + tuple(s), torch.float32, x.device) for s in layer_shapes]
+        ptrs = (C.c_void_p * len(net))(*[o.data_ptr() for o in outs])
+    _check(lib().dab_network_forward(net.records, len(net), N, Cc, H, W, _ptr(x), _ptr(y), _ptr(ws), need, ptrs, _stream(stream)),
+           "dab_network_forward")
+    return (y, outs) if keep_layers else y
