@@ -1,16 +1,21 @@
 """Stage-by-stage timings of libdab on the five synthetic workload configurations.
 
-`python -m paper_1804_02941_b200.sweep [--configs 1,2,3,4,5] [--batch5 256]` prints one JSON line per
+`python sweep.py [--configs 1,2,3,4,5,net] [--batch5 256]` prints one JSON line per
 (config, layer or point, stage): device time by CUDA events (best of a few repetitions after warm-up), the
 stage's throughput and its fraction of the relevant roofline (HBM copy bandwidth for binarize and pack; for the
 contraction, whichever kernel runs, alu_frac is its rate over the bound of the population-count kernel's
-instruction mix, so values above 1 are the tensor-core kernel beating the integer pipes).  bench.py is the benchmark of record; this is the wider table.
+instruction mix, so values above 1 are the tensor-core kernel beating the integer pipes).  `net` times whole networks
+(dab_network_forward: Sketch-A-Net-shaped at batch 1 = latency, AlexNet- and ResNet-18-shaped at batch 32).
+bench.py is the benchmark of record; this is the wider table.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 
 import numpy as np
 import torch
@@ -19,8 +24,8 @@ import dab_synth
 from dab_synth import configs
 import paper_1804_02941_b200 as dab
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-SM_COUNT, POPC_PER_CLK, WORDS_PER_POPC = 148, 16, 1.5
+ROOT = os.path.dirname(os.path.abspath(__file__))
+POPC_PER_CLK, WORDS_PER_POPC = 16, 1.5
 
 
 def peaks():
@@ -139,12 +144,22 @@ def pack_point(rows, n, hbm):
     emit(stage="pack", rows=rows, n=n, ms=t, gbs=b / t / 1e6, hbm_frac=b / t / 1e6 / hbm)
 
 
+def network_point(name, build, batch):
+    from dab_synth import networks
+    layers, shape = build()
+    net = dab.Network(layers)
+    x = torch.from_numpy(networks.network_input(shape, batch, stream=1)).cuda()
+    t = timed(lambda: dab.dab_network_forward(net, x), reps=5, warm=2)
+    emit(stage="network_forward", network=name, batch=batch, ms=t, images_per_s=batch / t * 1e3, layers=len(layers),
+         binarized_layers=sum(l["kind"] == "conv_binary" for l in layers))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--batch5", type=int, default=256)
     ap.add_argument("--contraction", default="auto", choices=["auto", "tensor", "popc"])
-    ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist"])
+    ap.add_argument("--patch-coder", default="auto", choices=["auto", "sort", "hist", "pixel"])
     ap.add_argument("--stages", default="", help="comma-separated stage names of the convolution layers to run (default all)")
     ap.add_argument("--layers", default="", help="comma-separated layer names to run (default all)")
     args = ap.parse_args()
@@ -152,13 +167,14 @@ def main():
     STAGES = set(args.stages.split(",")) if args.stages else None
     LAYERS = set(args.layers.split(",")) if args.layers else None
     dab.dab_set_contraction({"auto": dab.CONTRACT_AUTO, "tensor": dab.CONTRACT_TENSOR, "popc": dab.CONTRACT_POPC}[args.contraction])
-    dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST}[args.patch_coder])
+    dab.dab_set_patch_coder({"auto": dab.PATCHES_AUTO, "sort": dab.PATCHES_SORT, "hist": dab.PATCHES_HIST, "pixel": dab.PATCHES_PIXEL}[args.patch_coder])
     want = set(args.configs.split(","))
     hbm, mhz, src = peaks()
+    SM_COUNT = torch.cuda.get_device_properties(0).multi_processor_count
     tops_peak = POPC_PER_CLK * WORDS_PER_POPC * SM_COUNT * mhz * 1e6 * 64 / 1e12
     emit(contraction=args.contraction)
     emit(peaks=dict(hbm_gbs=hbm, source=src, contraction_tops_equiv=tops_peak,
-                    contraction_peak="16 popc/clk/SM x 1.5 words/popc x 148 SMs x %.0f MHz x 64" % mhz))
+                    contraction_peak="16 popc/clk/SM x 1.5 words/popc x %d SMs x %.0f MHz x 64" % (SM_COUNT, mhz)))
     if "1" in want:
         conv_layer(1, configs.config1()[0], 0, hbm, tops_peak)
     if "2" in want:
@@ -181,6 +197,11 @@ def main():
             seen.add(key)
             conv_layer(5, L, i, hbm, tops_peak)
         conv_layer(5, configs.config5(args.batch5)[0], 50, hbm, tops_peak, dense=True)
+    if "net" in want:
+        from dab_synth import networks
+        network_point("sketch_a_net", networks.sketch_a_net, 1)
+        network_point("alexnet_like", networks.alexnet_like, 32)
+        network_point("resnet18_like", networks.resnet18_like, 32)
 
 
 if __name__ == "__main__":
