@@ -440,8 +440,29 @@ def run_dab(args):
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
         e2e_s = max_over_ranks(e2e_s, world, dev)
+        # The floor the copies alone set: the same bytes per step moved by plain asynchronous copies from and to the
+        # same pinned buffers, both directions at once on two streams, nothing computed.
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        x_dev = {shape: torch.empty(shape, dtype=torch.float32, device=dev) for shape in host_x}
+
+        def copies_only():
+            for li, (L, x, w, wc, desc, pm, y) in enumerate(work):
+                with torch.cuda.stream(s_in):
+                    x_dev[L.x_shape()].copy_(host_x[L.x_shape()], non_blocking=True)
+                with torch.cuda.stream(s_out):
+                    y_hosts[li & 1][: L.patches * L.Cout].copy_(y_flat[: L.patches * L.Cout], non_blocking=True)
+        copies_only()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(3):
+            copies_only()
+        torch.cuda.synchronize()
+        floor_ms = 1e3 * (time.perf_counter() - t0) / 3
         e2e = {"value": aggregate_throughput(ops_per_step, args.e2e_steps, e2e_s, world) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * e2e_s / args.e2e_steps}
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * e2e_s / args.e2e_steps,
+               "pcie_floor_ms": floor_ms, "over_pcie_floor": 1e3 * e2e_s / args.e2e_steps / floor_ms,
+               "pcie_floor_note": "the step's %.2f GB in and %.2f GB out as plain pinned-memory copies on two streams at once, no "
+                                  "kernels: %.1f GB/s in, %.1f GB/s out" % (h2d / 1e9, d2h / 1e9, h2d / floor_ms / 1e6, d2h / floor_ms / 1e6)}
 
     # The paper's weights-only binarized networks on the same layers: fp32 activations against the coded filters
     # (dab_wbin_conv, four int8 tensor-core products per multiply-accumulate).  Reported beside the headline, not in it.

@@ -232,8 +232,8 @@ dab_status dab_binarize_backward(const float* d_Wc, int64_t rows, int32_t n, int
                                  float* d_grad_W, int64_t ld_grad_W, void* stream);
 
 /*
- * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into up
- * to 16 chunks of images; host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
+ * dab_binary_conv_host — the same layer for a caller whose tensors live in host memory.  The batch is cut into 2 to
+ * 16 chunks of images (of at least 8 MB where the batch allows); host-to-device copies, the kernels (on `stream`) and device-to-host copies of successive
  * chunks overlap on three streams, and the call returns after everything has drained.  Use pinned host memory:
  * with pageable memory the copies are staged by the driver and do not overlap.  The two copy streams and a few
  * events are created on the first call on a device and kept for the life of the process (the only state the
@@ -248,7 +248,10 @@ dab_status dab_binary_conv_host(const dab_conv_desc* desc, const float* h_x, con
 
 /*
  * dab_binary_conv_host_async — the same call without the final wait: it returns once all its copies and kernels
- * are queued, so that the next layer's copy-in overlaps this layer's last kernels and copy-out.  h_y is complete,
+ * are queued, so that the next layer's copy-in overlaps this layer's last kernels and copy-out.  Unlike
+ * dab_binary_conv_host, whose first copy waits for the work already queued on `stream`, this form starts copying
+ * h_x at once: h_x must hold its data when the call is made (the filters, device data, are still read in stream
+ * order).  h_y is complete,
  * and h_x, the filters and the workspace may be reused or freed, only after dab_binary_conv_host_wait (or a later
  * dab_binary_conv_host on the device) has returned.  A call whose workspace overlaps that of one of the last two
  * unfinished calls waits for it on the device, and at most two calls are left running at a time: give

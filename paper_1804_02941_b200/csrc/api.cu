@@ -253,7 +253,9 @@ dab_status dab_binary_conv_sign(const dab_conv_desc* desc, const float* d_x, con
 // ---------------------------------------------------------------------------------------------------------
 namespace {
 
-constexpr int kHostChunks = 16;  // chunks per call at most
+constexpr int kHostChunks = 16;                    // chunks per call at most
+constexpr size_t kHostChunkBytes = 32u << 20;      // and no smaller than this (of input or output, whichever is larger):
+                                                   // every chunk costs a fixed few tens of microseconds of launches and events
 
 struct HostPipe {
   bool ready = false;
@@ -303,10 +305,15 @@ struct HostPlan {
 };
 
 bool host_plan(const dab_conv_desc* desc, const ConvGeom& g, HostPlan* p) {
-  p->chunk_imgs = (desc->N + kHostChunks - 1) / kHostChunks;
-  p->chunks = (desc->N + p->chunk_imgs - 1) / p->chunk_imgs;
   p->x_img = (size_t)desc->C * desc->H * desc->W * sizeof(float);
   p->y_img = (size_t)desc->Cout * g.Ho * g.Wo * sizeof(float);
+  const size_t img_bytes = p->x_img > p->y_img ? p->x_img : p->y_img;
+  int64_t chunks = (int64_t)((img_bytes * (size_t)desc->N + kHostChunkBytes - 1) / kHostChunkBytes);
+  if (chunks > kHostChunks) chunks = kHostChunks;
+  if (chunks < 2) chunks = 2;                       // two at least, so that copies and kernels overlap at all
+  if (chunks > desc->N) chunks = desc->N;
+  p->chunk_imgs = (int32_t)((desc->N + chunks - 1) / chunks);
+  p->chunks = (desc->N + p->chunk_imgs - 1) / p->chunk_imgs;
   p->x_chunk = round_up(p->x_img * p->chunk_imgs, kAlign);
   p->y_chunk = round_up(p->y_img * p->chunk_imgs, kAlign);
   dab_conv_desc d = *desc;
@@ -347,8 +354,10 @@ static dab_status conv_host(bool drain, const dab_conv_desc* desc, const float* 
 
 #define DAB_TRY(call) do { if ((call) != cudaSuccess) { cudaStreamSynchronize(hp->in); cudaStreamSynchronize(hp->out); \
                            cudaStreamSynchronize(st); return DAB_ERR_CUDA; } } while (0)
-  DAB_TRY(cudaEventRecord(hp->start, st));  // work already queued on the caller's stream comes first
-  DAB_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+  if (drain) {  // work already queued on the caller's stream comes before the first copy
+    DAB_TRY(cudaEventRecord(hp->start, st));
+    DAB_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+  }  // (the queued form reads h_x as it is at the time of the call, so that its copies overlap the kernels before it)
   // earlier calls still running on a workspace that overlaps this one (or about to lose their record) come first
   HostPipe::Tail& slot = hp->tail[hp->next_tail];
   for (int i = 0; i < 2; ++i) {
