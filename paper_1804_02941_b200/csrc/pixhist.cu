@@ -462,10 +462,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
                 if (lane >= o) incl += t;
               }
               const int excl = incl - my_len;
+              // (no one-key-per-lane variant for the smallest hulls: the extra code costs more in instruction fetches
+              // than its shorter network saves)
               if (__shfl_sync(0xFFFFFFFFu, incl, KMAX - 1) != m_sub) {
                 retry = true;  // cannot happen; never trust a mismatch
-              } else if (m_sub <= 32) {
-                res = pix_gather_sort_select<1, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
               } else if (m_sub <= 64) {
                 res = pix_gather_sort_select<2, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
               } else if (m_sub <= 128) {
@@ -489,7 +489,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
               }
               __syncwarp();
               if (fill != m_sub) retry = true;  // cannot happen; never trust a mismatch
-              else if (m_sub <= 32) res = pix_sort_select<1, kTable>(scratch, m_sub, z_in, a.n, lane, rcp, base);
               else if (m_sub <= 64) res = pix_sort_select<2, kTable>(scratch, m_sub, z_in, a.n, lane, rcp, base);
               else if (m_sub <= 128) res = pix_sort_select<4, kTable>(scratch, m_sub, z_in, a.n, lane, rcp, base);
               else res = pix_sort_select<8, kTable>(scratch, m_sub, z_in, a.n, lane, rcp, base);
@@ -731,14 +730,14 @@ cudaError_t launch_pix(PixArgs& a, cudaStream_t stream, bool* applicable) {
   return launch_pix_minb<W, 1, BPL, KHW, ListT, kTable>(a, smem[0], stream);
 }
 
-// Reciprocal table for rows of fewer than 2048 values; 8-bit channel indices where the channel count allows (3 x 3
-// windows of such rows have at most 227 channels).
+// Reciprocal table for rows of fewer than 2048 values; 8-bit channel indices for up to 256 channels (3 x 3 windows;
+// the general kernel, which also takes whatever falls through here, has 16-bit ones).
 template <int BPL>
 cudaError_t launch_pix_for(PixArgs& a, cudaStream_t stream, bool* applicable) {
   constexpr bool kTable = BPL <= 2;
   if (a.d.kh == 3 && a.d.kw == 3) {
-    if constexpr (BPL <= 2) return launch_pix<BPL, 9, uint8_t, kTable>(a, stream, applicable);
-    else return launch_pix<BPL, 9, uint16_t, kTable>(a, stream, applicable);
+    if (a.d.C <= 256) return launch_pix<BPL, 9, uint8_t, kTable>(a, stream, applicable);
+    if constexpr (BPL >= 4) return launch_pix<BPL, 9, uint16_t, kTable>(a, stream, applicable);
   }
   return launch_pix<BPL, 0, uint16_t, kTable>(a, stream, applicable);
 }
@@ -771,6 +770,8 @@ cudaError_t launch_binarize_patches_pixhist(const dab_conv_desc& d, int32_t Ho, 
   if (a.n <= 256 || a.n > 8192 || d.kh * d.kw > 64) return cudaSuccess;
   cudaError_t e;
   // buckets by patch length: about n / 18, so that the two to four buckets that survive hold a few dozen values
+  // (measured against half and twice as many: fewer buckets leave hulls that are slow on inputs without zeros, more
+  // cost their tables in shared memory and their bounds per patch more than the smaller hulls save)
   if (a.n < 1024) e = launch_pix_for<1>(a, stream, applicable);
   else if (a.n < 2048) e = launch_pix_for<2>(a, stream, applicable);
   else if (a.n < 4096) e = launch_pix_for<4>(a, stream, applicable);
