@@ -694,6 +694,9 @@ cudaError_t launch_pix_minb(PixArgs& a, size_t smem, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+#ifndef DAB_PIX_WIDE_FROM_BPL
+#define DAB_PIX_WIDE_FROM_BPL 4   // buckets per lane from which a CTA has 16 warps instead of 8
+#endif
 #ifndef DAB_PIX_WARPS
 #define DAB_PIX_WARPS 8
 #endif
@@ -705,7 +708,9 @@ cudaError_t launch_pix_minb(PixArgs& a, size_t smem, cudaStream_t stream) {
 // 1.25 x the best of all.
 template <int BPL, int KHW, typename ListT, bool kTable>
 cudaError_t launch_pix(PixArgs& a, cudaStream_t stream, bool* applicable) {
-  constexpr int W = DAB_PIX_WARPS;
+  // rows of 2048 values and more leave room for one to three CTAs per SM only (tables, values and lists of a pixel
+  // take 3 to 6 KB): their CTAs get twice the warps
+  constexpr int W = BPL >= DAB_PIX_WIDE_FROM_BPL ? 2 * DAB_PIX_WARPS : DAB_PIX_WARPS;
   constexpr int kMostCtas = BPL <= DAB_PIX_FOUR_CTAS_UPTO_BPL ? 4 : 3;
   PixArgs cand[4] = {a, a, a, a};
   size_t smem[4] = {0, 0, 0, 0};
