@@ -25,7 +25,8 @@ EXPORTS = ("dab_status_string", "dab_words_per_row", "dab_default_ld", "dab_bina
            "dab_binary_conv_contract", "dab_sign_binarize", "dab_sign_patches", "dab_binary_conv_sign", "dab_binary_conv_host_workspace",
            "dab_binary_conv_host", "dab_binary_conv_static_capacity", "dab_binary_conv_static", "dab_popc_probe",
            "dab_set_contraction", "dab_get_contraction", "dab_contraction_wait_failures", "dab_wbin_conv", "dab_wbin_conv_workspace", "dab_binarize_train", "dab_binarize_backward", "dab_set_patch_coder", "dab_get_patch_coder", "dab_binary_conv_host_async", "dab_binary_conv_host_wait",
-           "dab_network_output_shape", "dab_network_workspace", "dab_network_forward")
+           "dab_network_output_shape", "dab_network_workspace", "dab_network_forward", "dab_debug_bounds_enabled",
+           "dab_debug_bounds_report")
 
 
 class DabError(RuntimeError):
@@ -39,6 +40,20 @@ class ConvDesc(C.Structure):
 
 
 _lib = None
+
+
+def use_library(path: str) -> None:
+    """Load the library from `path` instead of the in-tree libdab.so (e.g. the bounds-checking libdab_debug.so).
+    Only before the first call into the library."""
+    global LIB_PATH
+    if _lib is not None and os.path.abspath(path) != os.path.abspath(LIB_PATH):
+        raise RuntimeError("a library is already loaded from %s" % LIB_PATH)
+    LIB_PATH = path
+
+
+class BoundsReport(C.Structure):
+    _fields_ = [("violations", C.c_uint64), ("index", C.c_int64), ("extent", C.c_int64), ("file_hash", C.c_uint32),
+                ("line", C.c_int32)]
 
 
 def lib() -> C.CDLL:
@@ -74,6 +89,8 @@ def lib() -> C.CDLL:
         L.dab_binary_conv_static_capacity.argtypes = []
         L.dab_binary_conv_static.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.dab_popc_probe.argtypes = [vp, i32, i32, vp]
+        L.dab_debug_bounds_enabled.restype = i32
+        L.dab_debug_bounds_report.argtypes = [C.POINTER(BoundsReport), i32]
         L.dab_wbin_conv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
         L.dab_wbin_conv_workspace.restype = C.c_size_t
         L.dab_wbin_conv_workspace.argtypes = [vp]
@@ -451,6 +468,26 @@ def dab_popc_probe(blocks: int, iters: int, sink: torch.Tensor | None = None, st
         sink = torch.empty(blocks * 256, dtype=torch.int32, device="cuda")
     _check(lib().dab_popc_probe(_ptr(sink), blocks, iters, _stream(stream)), "dab_popc_probe")
     return sink
+
+
+def dab_debug_bounds_enabled() -> bool:
+    return bool(lib().dab_debug_bounds_enabled())
+
+
+def dab_debug_bounds_report(reset: bool = True) -> dict:
+    """Violations recorded by a library built with the index checks (DabError with status 2 from an ordinary one).
+    `file` is the name of the source file of the first violation, found by hashing the names under csrc/."""
+    r = BoundsReport()
+    _check(lib().dab_debug_bounds_report(C.byref(r), int(reset)), "dab_debug_bounds_report")
+    name = None
+    if r.violations:
+        for f in os.listdir(os.path.join(_HERE, "csrc")):
+            h = 2166136261
+            for ch in f.encode():
+                h = ((h ^ ch) * 16777619) & 0xFFFFFFFF
+            if h == r.file_hash:
+                name = f
+    return {"violations": int(r.violations), "index": int(r.index), "extent": int(r.extent), "file": name, "line": int(r.line)}
 
 
 CONTRACT_AUTO, CONTRACT_TENSOR, CONTRACT_POPC = 0, 1, 2

@@ -1,4 +1,7 @@
-"""Builds libdab.so (sm_100a) in-tree with nvcc.  `python -m paper_1804_02941_b200.build [--force] [--verbose]`."""
+"""Builds libdab.so (sm_100a) in-tree with nvcc.  `python -m paper_1804_02941_b200.build [--force] [--verbose]`.
+
+`--debug-bounds` builds libdab_debug.so instead: the same sources with -DDAB_DEBUG_BOUNDS, whose kernels check
+their global-memory indices (include/dab_debug.h)."""
 from __future__ import annotations
 
 import os
@@ -12,6 +15,8 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 OBJDIR = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdab.so")
+DEBUG_OBJDIR = os.path.join(HERE, "_build_debug")
+DEBUG_LIB = os.path.join(HERE, "libdab_debug.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--fmad=false",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
@@ -33,13 +38,14 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(f) for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
     """Compile every .cu under csrc/ for sm_100a and link them into one shared library."""
+    LIB, OBJDIR = (DEBUG_LIB, DEBUG_OBJDIR) if debug_bounds else (globals()["LIB"], globals()["OBJDIR"])
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
         return LIB
     os.makedirs(OBJDIR, exist_ok=True)
     nvcc = _nvcc()
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DDAB_DEBUG_BOUNDS"] if debug_bounds else [])
 
     def compile_one(src):
         obj = os.path.join(OBJDIR, os.path.basename(src)[:-3] + ".o")
@@ -62,4 +68,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

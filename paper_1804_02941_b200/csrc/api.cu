@@ -124,6 +124,7 @@ dab_status dab_binary_gemm(int64_t M, int64_t N, int32_t n, const uint32_t* d_A,
   g.B = d_B; g.ldb = ldb; g.KB = d_KB; g.alpha = d_alpha; g.beta = d_beta;
   g.C = d_C;
   g.map.inner = M; g.map.outer_stride = 0; g.map.row_stride = ldc; g.map.col_stride = 1;
+  g.c_extent = (M - 1) * ldc + N;
   g.p11 = d_p11; g.ldp = ldp;
   return from_cuda(contract(g, /*lanes_along_rows=*/false, static_cast<cudaStream_t>(stream)));
 }
@@ -198,6 +199,7 @@ dab_status dab_binary_conv_contract(const dab_conv_desc* desc, const uint32_t* d
   a.C = d_y;
   int64_t HoWo = (int64_t)g.Ho * g.Wo;
   a.map.inner = HoWo; a.map.outer_stride = (int64_t)desc->Cout * HoWo; a.map.row_stride = 1; a.map.col_stride = HoWo;
+  a.c_extent = (int64_t)desc->N * desc->Cout * HoWo;
   a.p11 = d_p11; a.ldp = desc->Cout;
   return from_cuda(contract(a, /*lanes_along_rows=*/true, static_cast<cudaStream_t>(stream)));
 }

@@ -12,7 +12,7 @@ __device__ __forceinline__ bool cta_has_marked_row(const int32_t* K_out, int64_t
   for (int64_t i = threadIdx.x;; i += blockDim.x) {
     const int64_t row = ((int64_t)blockIdx.x + (i / per_cta) * gridDim.x) * per_cta + i % per_cta;
     if (row >= rows) break;
-    any |= K_out[row] == kRowMark;
+    any |= K_out[DAB_IDX(row, rows)] == kRowMark;
   }
   return __syncthreads_or(any) != 0;
 }
@@ -37,12 +37,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
   __syncthreads();
 
   for (int64_t row = (int64_t)blockIdx.x * kWarpsPerCta + warp; row < rows; row += (int64_t)gridDim.x * kWarpsPerCta) {
-    if (marked_only && K_out[row] != kRowMark) continue;
+    if (marked_only && K_out[DAB_IDX(row, rows)] != kRowMark) continue;
     const float* v = values + row * ld_values;
-    auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
+    auto keyof = [v, n](int i) { return order_key(__ldg(v + DAB_IDX(i, n))); };
     uint32_t kreg[R];
     RowResult res = warp_code_row<R, kFull>(keyof, n, lane, scratch, rcp, kreg);
-    if (lane == 0) {
+    if (lane == 0 && DAB_IN_BOUNDS(row, rows)) {
       K_out[row] = res.K;
       alpha_out[row] = res.alpha;
       beta_out[row] = res.beta;
@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) binarize_rows_warp_kernel(
     }
     uint32_t mine = warp_mask_words<R, kFull>(kreg, n, lane, res);
     uint32_t* mrow = mask_out + row * (int64_t)ld_mask;
-    for (int w = lane; w < ld_mask; w += 32) mrow[w] = (w < 32) ? mine : 0u;
+    for (int w = lane; w < ld_mask; w += 32)
+      if (DAB_IN_BOUNDS(row * ld_mask + w, rows * ld_mask)) mrow[w] = (w < 32) ? mine : 0u;
   }
 }
 
@@ -80,19 +81,19 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_rows_group_kernel(
   }
 
   for (int64_t row = (int64_t)blockIdx.x * G + group; row < rows; row += (int64_t)gridDim.x * G) {
-    if (marked_only && K_out[row] != kRowMark) continue;  // the same for every thread of the group
+    if (marked_only && K_out[DAB_IDX(row, rows)] != kRowMark) continue;  // the same for every thread of the group
     const float* v = values + row * ld_values;
-    auto keyof = [v](int i) { return order_key(__ldg(v + i)); };
+    auto keyof = [v, n](int i) { return order_key(__ldg(v + DAB_IDX(i, n))); };
     uint32_t kreg[R];
     group_code_row<W, R, kFull, kTable>(keyof, n, tig, scratch, gs, bar_id, rcp, kreg);
     const RowResult res = gs->result;
-    if (tig == 0) {
+    if (tig == 0 && DAB_IN_BOUNDS(row, rows)) {
       K_out[row] = res.K;
       alpha_out[row] = res.alpha;
       beta_out[row] = res.beta;
       if (flags_out) flags_out[row] = res.flags;
     }
-    group_store_mask<W, R, kFull>(kreg, n, ld_mask, tig, res, mask_out + row * (int64_t)ld_mask);
+    group_store_mask<W, R, kFull>(kreg, n, ld_mask, tig, res, mask_out, row, rows);
     group_barrier(bar_id, 32 * W);  // gs->result is overwritten by the next row
   }
 }
@@ -158,7 +159,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kerne
     const float* v = values + row * ld_values;
     auto element = [v, n, lane](int k) {  // element of round k for this lane (+0.0 folds -0.0), 0.0 beyond the row
       const int i = k * 32 + lane;
-      return i < n ? __fadd_rn(__ldg(v + i), 0.0f) : 0.0f;
+      return i < n ? __fadd_rn(__ldg(v + DAB_IDX(i, n)), 0.0f) : 0.0f;
     };
     // pass 0: range and number of the non-zero values
     uint32_t kmin = kPadKey, kmax = 0u;
@@ -188,10 +189,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kerne
       retry = !hist_search<BPL>(sweep, n, qz, hist, scratch, rcp, lane, res);
     }
     if (retry) {
-      if (lane == 0) K_out[row] = kRowMark;
+      if (lane == 0 && DAB_IN_BOUNDS(row, rows)) K_out[row] = kRowMark;
       continue;
     }
-    if (lane == 0) {
+    if (lane == 0 && DAB_IN_BOUNDS(row, rows)) {
       K_out[row] = res.K;
       alpha_out[row] = res.alpha;
       beta_out[row] = res.beta;
@@ -210,9 +211,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 3) binarize_rows_hist_kerne
         const uint32_t word = __ballot_sync(0xFFFFFFFFu, keep && ((kb + kk) * 32 + lane < n) && ((x >= tv) != flip));
         if (kk == lane) mine = word;
       }
-      if (lane < kend) mrow[kb + lane] = mine;
+      if (lane < kend && DAB_IN_BOUNDS(row * ld_mask + kb + lane, rows * ld_mask)) mrow[kb + lane] = mine;
     }
-    for (int w = rounds + lane; w < ld_mask; w += 32) mrow[w] = 0u;
+    for (int w = rounds + lane; w < ld_mask; w += 32)
+      if (DAB_IN_BOUNDS(row * ld_mask + w, rows * ld_mask)) mrow[w] = 0u;
   }
 }
 

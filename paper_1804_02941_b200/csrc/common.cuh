@@ -4,7 +4,70 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "dab.h"
+
+// Checked indexing.  A build with -DDAB_DEBUG_BOUNDS compares every global-memory index its kernels form with the
+// extent of the array it addresses.  The first violation seen by the kernels of a translation unit is recorded
+// (source file as a hash of its name, line, index, extent) together with a count of all of them; a violating
+// store is skipped and a violating load reads element 0 instead.  dab_debug_bounds_report() collects the records.
+// In the ordinary build the two macros cost nothing: DAB_IN_BOUNDS is `true` and DAB_IDX is its first argument.
+#ifdef DAB_DEBUG_BOUNDS
+namespace dab {
+namespace dbg {
+
+struct Record {
+  unsigned long long count;  // violations since the last reset
+  long long index, extent;   // of the first one
+  unsigned int file, line;   // FNV-1a hash of the base name of its source file, and its line
+};
+
+__host__ __device__ constexpr unsigned int file_id(const char* path) {
+  const char* base = path;
+  for (const char* p = path; *p; ++p)
+    if (*p == '/') base = p + 1;
+  unsigned int h = 2166136261u;
+  for (const char* p = base; *p; ++p) h = (h ^ (unsigned char)*p) * 16777619u;
+  return h;
+}
+
+static __device__ Record tu_record;
+
+__device__ __forceinline__ bool in_bounds(long long index, long long extent, unsigned int file, unsigned int line) {
+  if (index >= 0 && index < extent) return true;
+  if (atomicAdd(&tu_record.count, 1ull) == 0ull) {
+    tu_record.index = index;
+    tu_record.extent = extent;
+    tu_record.file = file;
+    tu_record.line = line;
+  }
+  return false;
+}
+
+using Reader = cudaError_t (*)(Record* out, bool reset);
+void register_reader(Reader reader);  // device.cu
+
+static cudaError_t read_tu_record(Record* out, bool reset) {
+  cudaError_t e = cudaMemcpyFromSymbol(out, tu_record, sizeof(Record));
+  if (e == cudaSuccess && reset) {
+    const Record zero{};
+    e = cudaMemcpyToSymbol(tu_record, &zero, sizeof(Record));
+  }
+  return e;
+}
+static const bool tu_reader_registered = (register_reader(&read_tu_record), true);
+
+}  // namespace dbg
+}  // namespace dab
+#define DAB_IN_BOUNDS(index, extent)                                                                    \
+  ::dab::dbg::in_bounds((long long)(index), (long long)(extent),                                       \
+                        std::integral_constant<unsigned int, ::dab::dbg::file_id(__FILE__)>::value, __LINE__)
+#define DAB_IDX(index, extent) (DAB_IN_BOUNDS(index, extent) ? (index) : 0)
+#else
+#define DAB_IN_BOUNDS(index, extent) (true)
+#define DAB_IDX(index, extent) (index)
+#endif
 
 namespace dab {
 
@@ -75,6 +138,7 @@ struct GemmArgs {
   const float* beta;
   float* C;
   OutMap map;
+  int64_t c_extent;  // elements from C to the end of the output it addresses (last offset of the map + 1)
   int32_t* p11;
   int64_t ldp;
 };

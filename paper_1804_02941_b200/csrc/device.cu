@@ -3,8 +3,10 @@
 // Both caches are guarded by one mutex; they hold nothing that a later call depends on for correctness.
 #include <mutex>
 #include <unordered_map>
+#include <vector>
 
 #include "common.cuh"
+#include "dab_debug.h"
 
 namespace dab {
 
@@ -41,3 +43,49 @@ cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
 }
 
 }  // namespace dab
+
+// Bounds report of the debug build: the per-translation-unit records of common.cuh, added up.
+#ifdef DAB_DEBUG_BOUNDS
+namespace dab {
+namespace dbg {
+namespace {
+std::vector<Reader>& readers() {
+  static std::vector<Reader> list;  // filled by static initialisers of the other translation units
+  return list;
+}
+}  // namespace
+void register_reader(Reader reader) { readers().push_back(reader); }
+}  // namespace dbg
+}  // namespace dab
+#endif
+
+extern "C" int32_t dab_debug_bounds_enabled(void) {
+#ifdef DAB_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+extern "C" dab_status dab_debug_bounds_report(dab_bounds_report* h_report, int32_t reset) {
+  if (h_report == nullptr) return DAB_ERR_INVALID_ARG;
+  *h_report = dab_bounds_report{};
+#ifdef DAB_DEBUG_BOUNDS
+  if (cudaDeviceSynchronize() != cudaSuccess) return DAB_ERR_CUDA;
+  for (dab::dbg::Reader read : dab::dbg::readers()) {
+    dab::dbg::Record r;
+    if (read(&r, reset != 0) != cudaSuccess) return DAB_ERR_CUDA;
+    if (r.count != 0 && h_report->violations == 0) {
+      h_report->index = r.index;
+      h_report->extent = r.extent;
+      h_report->file_hash = r.file;
+      h_report->line = (int32_t)r.line;
+    }
+    h_report->violations += r.count;
+  }
+  return DAB_OK;
+#else
+  (void)reset;
+  return DAB_ERR_UNSUPPORTED;
+#endif
+}

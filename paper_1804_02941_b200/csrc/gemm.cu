@@ -46,8 +46,10 @@ __global__ void __launch_bounds__(GEMM_THREADS) binary_gemm_kernel(const GemmArg
       const int r = t / (BK / 4), q = (t % (BK / 4)) * 4;
       uint4 qa = make_uint4(0, 0, 0, 0), qb = make_uint4(0, 0, 0, 0);
       if (k0 + q < g.words) {
-        if (i0 + r < g.M) qa = *reinterpret_cast<const uint4*>(g.A + (i0 + r) * (int64_t)g.lda + k0 + q);
-        if (j0 + r < g.N) qb = *reinterpret_cast<const uint4*>(g.B + (j0 + r) * (int64_t)g.ldb + k0 + q);
+        if (i0 + r < g.M)
+          qa = *reinterpret_cast<const uint4*>(g.A + DAB_IDX((i0 + r) * (int64_t)g.lda + k0 + q, g.M * g.lda - 3));
+        if (j0 + r < g.N)
+          qb = *reinterpret_cast<const uint4*>(g.B + DAB_IDX((j0 + r) * (int64_t)g.ldb + k0 + q, g.N * g.ldb - 3));
       }
       As[q + 0][r] = qa.x; As[q + 1][r] = qa.y; As[q + 2][r] = qa.z; As[q + 3][r] = qa.w;
       Bs[q + 0][r] = qb.x; Bs[q + 1][r] = qb.y; Bs[q + 2][r] = qb.z; Bs[q + 3][r] = qb.w;
@@ -85,24 +87,25 @@ __global__ void __launch_bounds__(GEMM_THREADS) binary_gemm_kernel(const GemmArg
   for (int j = 0; j < TN; ++j) {
     int64_t gj = j0 + b_t * TN + j;
     const bool in = gj < g.N;
-    al[j] = in ? (double)g.alpha[gj] : 0.0;
-    be[j] = in ? (double)g.beta[gj] : 0.0;
-    Ke[j] = in ? g.KB[gj] : 0;
+    al[j] = in ? (double)g.alpha[DAB_IDX(gj, g.N)] : 0.0;
+    be[j] = in ? (double)g.beta[DAB_IDX(gj, g.N)] : 0.0;
+    Ke[j] = in ? g.KB[DAB_IDX(gj, g.N)] : 0;
   }
 #pragma unroll
   for (int i = 0; i < TM; ++i) {
     int64_t gi = i0 + a_t * TM + i;
     if (gi >= g.M) continue;
-    int Kf = g.KA[gi];
-    double gam = (double)g.gamma[gi], del = (double)g.delta[gi];
+    int Kf = g.KA[DAB_IDX(gi, g.M)];
+    double gam = (double)g.gamma[DAB_IDX(gi, g.M)], del = (double)g.delta[DAB_IDX(gi, g.M)];
     int64_t base = (gi / g.map.inner) * g.map.outer_stride + (gi % g.map.inner) * g.map.row_stride;
 #pragma unroll
     for (int j = 0; j < TN; ++j) {
       int64_t gj = j0 + b_t * TN + j;
       if (gj >= g.N) continue;
       int p11 = ones[i][j] + 2 * twos[i][j];
-      g.C[base + gj * g.map.col_stride] = rescale(p11, Ke[j], Kf, g.n, al[j], be[j], gam, del);
-      if (g.p11) g.p11[gi * g.ldp + gj] = p11;
+      if (DAB_IN_BOUNDS(base + gj * g.map.col_stride, g.c_extent))
+        g.C[base + gj * g.map.col_stride] = rescale(p11, Ke[j], Kf, g.n, al[j], be[j], gam, del);
+      if (g.p11 && DAB_IN_BOUNDS(gi * g.ldp + gj, (g.M - 1) * g.ldp + g.N)) g.p11[gi * g.ldp + gj] = p11;
     }
   }
 }

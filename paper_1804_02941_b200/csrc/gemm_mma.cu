@@ -99,9 +99,9 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
   };
   for (int j = tid; j < nrows; j += THREADS) {
     ColumnParams cp;
-    const int K = S.K[j0 + j];
-    cp.v1 = (double)S.v1[j0 + j];
-    cp.v0 = (double)S.v0[j0 + j];
+    const int K = S.K[DAB_IDX(j0 + j, S.rows)];
+    cp.v1 = (double)S.v1[DAB_IDX(j0 + j, S.rows)];
+    cp.v0 = (double)S.v0[DAB_IDX(j0 + j, S.rows)];
     cp.K = (double)K;
     cp.nK = (double)(g.n - K);
     cp.off = kLanesAreActivations ? (j0 + j) * g.map.col_stride : act_offset(j0 + j);
@@ -133,9 +133,11 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
       const int w = w0 + 4 * piece;
       if (w >= g.words) continue;
       if (isL) {
-        if (i0 + row < L.rows) q[t] = *reinterpret_cast<const uint4*>(L.mask + (i0 + row) * (int64_t)L.ld + w);
+        if (i0 + row < L.rows)
+          q[t] = *reinterpret_cast<const uint4*>(L.mask + DAB_IDX((i0 + row) * (int64_t)L.ld + w, L.rows * L.ld - 3));
       } else {
-        if (row < nrows) q[t] = *reinterpret_cast<const uint4*>(S.mask + (j0 + row) * (int64_t)S.ld + w);
+        if (row < nrows)
+          q[t] = *reinterpret_cast<const uint4*>(S.mask + DAB_IDX((j0 + row) * (int64_t)S.ld + w, S.rows * S.ld - 3));
       }
     }
   };
@@ -183,9 +185,9 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
     double Kl = 0.0, l1 = 0.0, l0 = 0.0;
     int64_t off = 0;
     if (valid) {
-      Kl = (double)L.K[gl];
-      l1 = (double)L.v1[gl];
-      l0 = (double)L.v0[gl];
+      Kl = (double)L.K[DAB_IDX(gl, L.rows)];
+      l1 = (double)L.v1[DAB_IDX(gl, L.rows)];
+      l0 = (double)L.v0[DAB_IDX(gl, L.rows)];
       off = kLanesAreActivations ? act_offset(gl) : gl * g.map.col_stride;
     }
     for (int cb = warp >> 2; cb * 32 < NT; cb += THREADS / 128) {
@@ -212,8 +214,9 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
           y = __dadd_rn(y, __dmul_rn(__dmul_rn(l0, cp.v1), pc));
         }
         y = __dadd_rn(y, __dmul_rn(__dmul_rn(cp.v0, l0), p00));
-        g.C[off + cp.off] = (float)y;
-        if (g.p11) g.p11[kLanesAreActivations ? gl * g.ldp + j0 + j : (j0 + j) * g.ldp + gl] = (int)v[jj];
+        if (DAB_IN_BOUNDS(off + cp.off, g.c_extent)) g.C[off + cp.off] = (float)y;
+        const int64_t pidx = kLanesAreActivations ? gl * g.ldp + j0 + j : (j0 + j) * g.ldp + gl;
+        if (g.p11 && DAB_IN_BOUNDS(pidx, (g.M - 1) * g.ldp + g.N)) g.p11[pidx] = (int)v[jj];
       }
     }
   }

@@ -27,17 +27,20 @@ __global__ void __launch_bounds__(256) pack_aligned_kernel(const uint8_t* __rest
     uint32_t w = t - row * (uint32_t)ld_mask;
     if (w >= (uint32_t)ld_mask) { w -= ld_mask; ++row; }
     const int e0 = (int)w * 32;
-    const uint8_t* b = bits + (row_begin + row) * ld_bits + e0;
+    const int64_t bit_extent = (row_begin + rows - 1) * ld_bits + n;  // bytes up to the end of this launch's last row
+    const int64_t b0 = (row_begin + row) * ld_bits + e0;
+    const uint8_t* b = bits + b0;
     uint32_t word = 0;
     if (e0 + 32 <= n) {
-      const uint4 q0 = __ldg(reinterpret_cast<const uint4*>(b));
-      const uint4 q1 = __ldg(reinterpret_cast<const uint4*>(b) + 1);
+      const uint4 q0 = __ldg(reinterpret_cast<const uint4*>(bits + DAB_IDX(b0, bit_extent - 15)));
+      const uint4 q1 = __ldg(reinterpret_cast<const uint4*>(bits + DAB_IDX(b0 + 16, bit_extent - 15)));
       word = bits16_of(q0) | (bits16_of(q1) << 16);
     } else if (e0 < n) {  // the one ragged word of a row; words past the row stay 0
       for (int k = 0; k < n - e0; ++k)
-        if (b[k]) word |= 1u << k;
+        if (b[DAB_IDX(k, bit_extent - b0)]) word |= 1u << k;
     }
-    mask[(row_begin + row) * (int64_t)ld_mask + w] = word;
+    if (DAB_IN_BOUNDS((row_begin + row) * (int64_t)ld_mask + w, (row_begin + rows) * (int64_t)ld_mask))
+      mask[(row_begin + row) * (int64_t)ld_mask + w] = word;
   }
 }
 
@@ -49,10 +52,10 @@ __global__ void __launch_bounds__(256) count_ones_thread_kernel(const uint32_t* 
     const uint4* m = reinterpret_cast<const uint4*>(mask + row * (int64_t)ld_mask);
     int c = 0;
     for (int q = 0; q < ld_mask / 4; ++q) {
-      const uint4 v = __ldg(m + q);
+      const uint4 v = __ldg(m + DAB_IDX(q, ld_mask / 4));
       c += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
     }
-    K[row] = c;
+    if (DAB_IN_BOUNDS(row, rows)) K[row] = c;
   }
 }
 
@@ -63,9 +66,9 @@ __global__ void __launch_bounds__(256) count_ones_warp_kernel(const uint32_t* __
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   for (int64_t row = warp0; row < rows; row += nwarps) {
     int c = 0;
-    for (int w = lane; w < ld_mask; w += 32) c += __popc(mask[row * (int64_t)ld_mask + w]);
+    for (int w = lane; w < ld_mask; w += 32) c += __popc(mask[DAB_IDX(row * (int64_t)ld_mask + w, rows * ld_mask)]);
     c = __reduce_add_sync(0xFFFFFFFFu, c);
-    if (lane == 0) K[row] = c;
+    if (lane == 0 && DAB_IN_BOUNDS(row, rows)) K[row] = c;
   }
 }
 
@@ -83,12 +86,12 @@ __global__ void __launch_bounds__(256) pack_bytes_kernel(const uint8_t* __restri
     int count = 0;
     for (int w = 0; w < ld_mask; ++w) {
       int i = w * 32 + lane;
-      bool bit = i < n && b[i] != 0;
+      bool bit = i < n && b[DAB_IDX(i, n)] != 0;
       uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
-      if (lane == 0) m[w] = word;
+      if (lane == 0 && DAB_IN_BOUNDS(row * ld_mask + w, rows * ld_mask)) m[w] = word;
       count += __popc(word);
     }
-    if (K && lane == 0) K[row] = count;
+    if (K && lane == 0 && DAB_IN_BOUNDS(row, rows)) K[row] = count;
   }
 }
 

@@ -35,6 +35,10 @@ struct PatchArgs {
   int32_t ldp;
 };
 
+// Extents of the arrays of a call (what the checked indices of a debug build are compared with).
+__device__ __forceinline__ int64_t patch_count(const PatchArgs& a) { return (int64_t)a.d.N * a.Ho * a.Wo; }
+__device__ __forceinline__ int64_t image_values(const PatchArgs& a) { return (int64_t)a.d.C * a.d.H * a.d.W; }
+
 __device__ __forceinline__ void fill_offsets(const PatchArgs& a, uint16_t* off, int ch_words, int tid, int threads) {
   const int khw = a.d.kh * a.d.kw;
   for (int i = tid; i < a.n; i += threads) {
@@ -60,7 +64,7 @@ __device__ __forceinline__ int load_tile(const PatchArgs& a, const float* __rest
     int h = h0 + r, w = w0 + s;
     float v = 0.0f;
     if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
-      v = __ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w);
+      v = __ldg(ximg + DAB_IDX(((int64_t)c * a.d.H + h) * a.d.W + w, image_values(a)));
     tile[c * ch_words + r * a.pitch + s] = kKeys ? __uint_as_float(order_key(v)) : v;
     nonzero += (v != 0.0f);
   }
@@ -103,7 +107,7 @@ __device__ __forceinline__ bool has_marked_tile(const PatchArgs& a) {
   for (int64_t tile_id = blockIdx.x + (int64_t)threadIdx.x * gridDim.x; tile_id < total_tiles;
        tile_id += (int64_t)blockDim.x * gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
-    any |= a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] == kDenseMark;
+    any |= a.pK[DAB_IDX(((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0, patch_count(a))] == kDenseMark;
   }
   return __syncthreads_or(any) != 0;
 }
@@ -146,7 +150,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
       __syncthreads();
       const int64_t staged = staged_inside(a, t);
       if ((int64_t)tile_nonzero * a.dense_den > a.dense_num * staged) {
-        if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+        if (threadIdx.x == 0 && DAB_IN_BOUNDS(first_patch, patch_count(a))) a.pK[first_patch] = kDenseMark;
         continue;
       }
     } else {
@@ -160,7 +164,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
       uint32_t kreg[R];
       RowResult res = warp_code_row<R, kFull>(keyof, a.n, lane, scratch, rcp, kreg);
       const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
-      if (lane == 0) {
+      if (lane == 0 && DAB_IN_BOUNDS(pi, patch_count(a))) {
         a.pK[pi] = res.K;
         a.pgamma[pi] = res.alpha;
         a.pdelta[pi] = res.beta;
@@ -168,7 +172,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_WARP_MINBLOCKS) binariz
       }
       uint32_t mine = warp_mask_words<R, kFull>(kreg, a.n, lane, res);
       uint32_t* mrow = a.pmask + pi * (int64_t)a.ldp;
-      for (int w = lane; w < a.ldp; w += 32) mrow[w] = (w < 32) ? mine : 0u;
+      for (int w = lane; w < a.ldp; w += 32)
+        if (DAB_IN_BOUNDS(pi * a.ldp + w, patch_count(a) * a.ldp)) mrow[w] = (w < 32) ? mine : 0u;
     }
   }
 }
@@ -199,7 +204,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
     const int64_t first_patch = ((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0;
-    if (a.marked_only && a.pK[first_patch] != kDenseMark) continue;
+    if (a.marked_only && a.pK[DAB_IDX(first_patch, patch_count(a))] != kDenseMark) continue;
     __syncthreads();
     if (threadIdx.x == 0) tile_nonzero = 0;
     int nz = load_tile<true>(a, a.x + (int64_t)t.img * a.d.C * a.d.H * a.d.W, t.h0, t.w0, tile, ch_words, threadIdx.x,
@@ -211,7 +216,7 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
       __syncthreads();
       const int64_t staged = staged_inside(a, t);
       if ((int64_t)tile_nonzero * a.dense_den > a.dense_num * staged) {
-        if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+        if (threadIdx.x == 0 && DAB_IN_BOUNDS(first_patch, patch_count(a))) a.pK[first_patch] = kDenseMark;
         continue;
       }
     }
@@ -224,13 +229,13 @@ __global__ void __launch_bounds__(WARPS * 32) binarize_patches_group_kernel(cons
       group_code_row<W, R, kFull, kTable>(keyof, a.n, tig, scratch, gs, bar_id, rcp, kreg);
       const RowResult res = gs->result;
       const int64_t pi = ((int64_t)t.img * a.Ho + (t.ho0 + lh)) * a.Wo + (t.wo0 + lw);
-      if (tig == 0) {
+      if (tig == 0 && DAB_IN_BOUNDS(pi, patch_count(a))) {
         a.pK[pi] = res.K;
         a.pgamma[pi] = res.alpha;
         a.pdelta[pi] = res.beta;
         if (a.pflags) a.pflags[pi] = res.flags;
       }
-      group_store_mask<W, R, kFull>(kreg, a.n, a.ldp, tig, res, a.pmask + pi * (int64_t)a.ldp);
+      group_store_mask<W, R, kFull>(kreg, a.n, a.ldp, tig, res, a.pmask, pi, patch_count(a));
       group_barrier(bar_id, 32 * W);
     }
   }
@@ -286,7 +291,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
   const int64_t total_tiles = (int64_t)a.tiles_h * a.tiles_w * a.d.N;
   for (int64_t tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
     const TileCoord t = tile_coord(a, tile_id);
-    if (a.marked_only && a.pK[((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0] != kDenseMark) continue;
+    if (a.marked_only && a.pK[DAB_IDX(((int64_t)t.img * a.Ho + t.ho0) * a.Wo + t.wo0, patch_count(a))] != kDenseMark) continue;
     __syncthreads();  // the previous tile is no longer read
     if (threadIdx.x == 0) { ht.kmin = kPadKey; ht.kmax = 0u; ht.retry = 0; }
     __syncthreads();
@@ -302,7 +307,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
         int h = t.h0 + r, w = t.w0 + s;
         float v = 0.0f;
         if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
-          v = __fadd_rn(__ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w), 0.0f);
+          v = __fadd_rn(__ldg(ximg + DAB_IDX(((int64_t)c * a.d.H + h) * a.d.W + w, image_values(a))), 0.0f);
         tile[c * ch_words + r * a.pitch + s] = v;
         if (v != 0.0f) {  // NaN compares unequal: counted, and seen as non-finite below
           const uint32_t key = order_key(v);
@@ -322,7 +327,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
     const uint32_t tkmin = ht.kmin, tkmax = ht.kmax;
     const bool any_nonzero = tkmin <= tkmax;
     if (any_nonzero && key_range_nonfinite(tkmin, tkmax)) {
-      if (threadIdx.x == 0) a.pK[first_patch] = kDenseMark;
+      if (threadIdx.x == 0 && DAB_IN_BOUNDS(first_patch, patch_count(a))) a.pK[first_patch] = kDenseMark;
       continue;
     }
     const float lo = any_nonzero ? key_value(tkmin) : 0.0f, hi = any_nonzero ? key_value(tkmax) : 0.0f;
@@ -354,7 +359,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
         continue;
       }
       // ---- pass 3: outputs (mask bits in element order, through the offset table) ----
-      if (lane == 0) {
+      if (lane == 0 && DAB_IN_BOUNDS(pi, patch_count(a))) {
         a.pK[pi] = res.K;
         a.pgamma[pi] = res.alpha;
         a.pdelta[pi] = res.beta;
@@ -374,12 +379,13 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, DAB_HIST_MINBLOCKS) binariz
           const uint32_t word = __ballot_sync(0xFFFFFFFFu, keep && live && ((v >= tv) != flip));
           if (kk == lane) mine = word;
         }
-        if (lane < kend) mrow[kb + lane] = mine;
+        if (lane < kend && DAB_IN_BOUNDS(pi * a.ldp + kb + lane, patch_count(a) * a.ldp)) mrow[kb + lane] = mine;
       }
-      for (int w = rounds + lane; w < a.ldp; w += 32) mrow[w] = 0u;
+      for (int w = rounds + lane; w < a.ldp; w += 32)
+        if (DAB_IN_BOUNDS(pi * a.ldp + w, patch_count(a) * a.ldp)) mrow[w] = 0u;
     }
     __syncthreads();
-    if (threadIdx.x == 0 && ht.retry) a.pK[first_patch] = kDenseMark;
+    if (threadIdx.x == 0 && ht.retry && DAB_IN_BOUNDS(first_patch, patch_count(a))) a.pK[first_patch] = kDenseMark;
   }
 }
 

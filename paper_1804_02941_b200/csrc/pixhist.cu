@@ -53,6 +53,9 @@ struct PixArgs {
   int32_t ldp;
 };
 
+// Patches of the call: the extent of pK, pgamma, pdelta and pflags (and, times ldp, of pmask).
+__device__ __forceinline__ int64_t patch_count(const PixArgs& a) { return (int64_t)a.d.N * a.Ho * a.Wo; }
+
 // Bucket grid of a tile: bucket(v) = floor(v * 2^k) + B0 for the non-zero values v, with k the largest exponent
 // that keeps every value of the tile inside the B buckets.  Multiplying by a power of two is exact, so bucket b
 // holds exactly the values in [(b - B0) 2^-k, (b - B0 + 1) 2^-k).
@@ -219,12 +222,11 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
       for (int p = lane; p < pixn; p += 32) {
         const int o = poff[p];
         if (o >= 0) {
-          const float* src = ximg + o;
           const unsigned saddr = (unsigned)__cvta_generic_to_shared(tile + p);
 #pragma unroll kPixUnroll
           for (int c = warp; c < C; c += WARPS)
             asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(saddr + 4u * (unsigned)(c * chw)),
-                         "l"(src + (int64_t)c * plane) : "memory");
+                         "l"(ximg + DAB_IDX(o + (int64_t)c * plane, (int64_t)C * plane)) : "memory");
         } else {
           for (int c = warp; c < C; c += WARPS) tile[c * chw + p] = 0.0f;
         }
@@ -257,7 +259,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     PixQuant qz = make_pix_quant(any_nonzero ? tkmin : kZeroKey + 1u, any_nonzero ? tkmax : kZeroKey + 1u, LOG2B);
     if (any_nonzero && (key_range_nonfinite(tkmin, tkmax) || !qz.ok)) {
       // every patch of the tile is left to the sorting kernel
-      for (int p = threadIdx.x; p < npatch; p += THREADS) a.pK[tile_base + (int64_t)(p / tw) * a.Wo + p % tw] = kRowMark;
+      for (int p = threadIdx.x; p < npatch; p += THREADS) {
+        const int64_t pi = tile_base + (int64_t)(p / tw) * a.Wo + p % tw;
+        if (DAB_IN_BOUNDS(pi, patch_count(a))) a.pK[pi] = kRowMark;
+      }
       continue;
     }
     // ---- per pixel: count and fp64 sum per bucket ----
@@ -507,10 +512,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
         }
       }
       if (retry) {
-        if (lane == 0) a.pK[pi] = kRowMark;
+        if (lane == 0 && DAB_IN_BOUNDS(pi, patch_count(a))) a.pK[pi] = kRowMark;
         continue;
       }
-      if (lane == 0) {
+      if (lane == 0 && DAB_IN_BOUNDS(pi, patch_count(a))) {
         a.pK[pi] = res.K;
         a.pgamma[pi] = res.alpha;
         a.pdelta[pi] = res.beta;
@@ -548,9 +553,11 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
           const uint32_t own = __shfl_sync(0xFFFFFFFFu, lo, first_of_word);
           const uint32_t spill = __shfl_sync(0xFFFFFFFFu, hi, first_of_prev);
           const int w = g * 9 + lane;
-          if (lane < 9 && w < a.ldp) mrow[w] = own | (lane ? spill : 0u);
+          if (lane < 9 && w < a.ldp && DAB_IN_BOUNDS(pi * a.ldp + w, patch_count(a) * a.ldp))
+            mrow[w] = own | (lane ? spill : 0u);
         }
-        for (int w = groups * 9 + lane; w < a.ldp; w += 32) mrow[w] = 0u;
+        for (int w = groups * 9 + lane; w < a.ldp; w += 32)
+          if (DAB_IN_BOUNDS(pi * a.ldp + w, patch_count(a) * a.ldp)) mrow[w] = 0u;
       } else {
         for (int kb = 0; kb < rounds; kb += 32) {  // 32 mask words at a time: word kb + j ends up in lane j
           const int kend = min(32, rounds - kb);
@@ -562,9 +569,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
             const uint32_t word = __ballot_sync(0xFFFFFFFFu, !none && live && ((v >= tv) != flip));
             if (kk == lane) mine = word;
           }
-          if (lane < kend) mrow[kb + lane] = mine;
+          if (lane < kend && DAB_IN_BOUNDS(pi * a.ldp + kb + lane, patch_count(a) * a.ldp)) mrow[kb + lane] = mine;
         }
-        for (int w = rounds + lane; w < a.ldp; w += 32) mrow[w] = 0u;
+        for (int w = rounds + lane; w < a.ldp; w += 32)
+          if (DAB_IN_BOUNDS(pi * a.ldp + w, patch_count(a) * a.ldp)) mrow[w] = 0u;
       }
     }
   }
@@ -590,7 +598,7 @@ __global__ void __launch_bounds__(kFixThreads) binarize_patches_fixup_kernel(con
     __syncthreads();
     if (tig == 0) qn = 0;
     __syncthreads();
-    if (chunk + tig < total && a.pK[chunk + tig] == kRowMark) queue[atomicAdd(&qn, 1)] = tig;
+    if (chunk + tig < total && a.pK[DAB_IDX(chunk + tig, total)] == kRowMark) queue[atomicAdd(&qn, 1)] = tig;
     __syncthreads();
     const int count = qn;
     for (int qi = 0; qi < count; ++qi) {
@@ -606,19 +614,19 @@ __global__ void __launch_bounds__(kFixThreads) binarize_patches_fixup_kernel(con
         const int h = hb + r, w = wb + s;
         float v = 0.0f;
         if ((unsigned)h < (unsigned)a.d.H && (unsigned)w < (unsigned)a.d.W)
-          v = __ldg(ximg + ((int64_t)c * a.d.H + h) * a.d.W + w);
+          v = __ldg(ximg + DAB_IDX(((int64_t)c * a.d.H + h) * a.d.W + w, (int64_t)a.d.C * a.d.H * a.d.W));
         return order_key(v);
       };
       uint32_t kreg[R];
       group_code_row<W, R, false, false>(keyof, a.n, tig, scratch, gs, 1, nullptr, kreg);
       const RowResult res = gs->result;
-      if (tig == 0) {
+      if (tig == 0 && DAB_IN_BOUNDS(pi, total)) {
         a.pK[pi] = res.K;
         a.pgamma[pi] = res.alpha;
         a.pdelta[pi] = res.beta;
         if (a.pflags) a.pflags[pi] = res.flags;
       }
-      group_store_mask<W, R, false>(kreg, a.n, a.ldp, tig, res, a.pmask + pi * (int64_t)a.ldp);
+      group_store_mask<W, R, false>(kreg, a.n, a.ldp, tig, res, a.pmask, pi, total);
       group_barrier(1, 32 * W);  // gs->result is overwritten by the next patch
     }
   }

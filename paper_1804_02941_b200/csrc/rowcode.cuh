@@ -547,11 +547,14 @@ __device__ __forceinline__ void group_code_row(KeyOf keyof, int n, int tig, uint
   group_barrier(bar_id, GT);
 }
 
-// Mask words of a row coded by a group: warp w produces words w*R .. w*R+R-1 (word w*R+k in lane k) and stores
-// them with one coalesced write; words from W*R up to ld are written as 0.
+// Mask words of row `row` (of `rows`, ld words each, starting at `masks`) coded by a group: warp w produces words
+// w*R .. w*R+R-1 (word w*R+k in lane k) and stores them with one coalesced write; words from W*R up to ld are
+// written as 0.
 template <int W, int R, bool kFull>
 __device__ __forceinline__ void group_store_mask(const uint32_t (&kreg)[R], int n, int ld, int tig,
-                                                 const RowResult& res, uint32_t* __restrict__ out) {
+                                                 const RowResult& res, uint32_t* __restrict__ masks, int64_t row,
+                                                 int64_t rows) {
+  uint32_t* const out = masks + row * (int64_t)ld;
   const int lane = tig & 31, warp = tig >> 5;
   const bool flip = res.mode == 1;
   uint32_t mine = 0;
@@ -563,8 +566,9 @@ __device__ __forceinline__ void group_store_mask(const uint32_t (&kreg)[R], int 
     if (lane == k) mine = word;
   }
   const int w = warp * R + lane;
-  if (lane < R && w < ld) out[w] = mine;
-  for (int p = W * R + tig; p < ld; p += 32 * W) out[p] = 0u;
+  if (lane < R && w < ld && DAB_IN_BOUNDS(row * ld + w, rows * ld)) out[w] = mine;
+  for (int p = W * R + tig; p < ld; p += 32 * W)
+    if (DAB_IN_BOUNDS(row * ld + p, rows * ld)) out[p] = 0u;
 }
 
 // ---------------------------------------------------------------------------------------------------------
