@@ -1,8 +1,9 @@
 // Tensor-core form of the AND-popcount contraction (Section 4.2: the four population counts of a pair of
 // coded rows).  popc(e AND f) over a row of n bits is the dot product of the two rows written as 0/1 bytes,
 // so each CTA expands mask words to bytes in shared memory and lets the fifth-generation tensor cores
-// (tcgen05.mma, kind::i8, unsigned 8-bit operands, 32-bit integer accumulators in tensor memory) form a
-// 128 x NT block of exact integer counts.  The four-term rescale then runs on the counts as they are read
+// (tcgen05.mma, kind::i8, 32-bit integer accumulators in tensor memory) form a 128 x NT block of exact integer
+// counts.  The bytes are 0 / -1 (signed operands on both sides: one byte permutation per four bits makes them,
+// and (-1) x (-1) = 1), in an order of the row's bits that is permuted within each word, alike on both sides.  The four-term rescale then runs on the counts as they are read
 // back from tensor memory, with the same arithmetic as the population-count kernel.
 //
 // Shared-memory operand layout (K-major, no swizzle): 8 rows x 16 bytes form one contiguous 128-byte core
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = s_tmem;
-  const uint32_t idesc = instr_desc(NT);
+  const uint32_t idesc = instr_desc(NT, true, true);  // both operands signed: bytes 0 / -1
 
   // units of this thread: lane-side pieces first, then column-side pieces
   const int l_units = MMA_M * KQ, units = l_units + NT * KQ;
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
       if (c * 4 * KQ + 4 * piece >= g.words) continue;  // no instruction reads this part of the stage
       unsigned char* dst =
           stage + (isL ? 0u : a_bytes) + (uint32_t)group * SBO + (uint32_t)(8 * piece) * 128 + (v & 7) * 16;
-      expand_words(q[t], dst);
+      expand_words_signed(q[t], dst);
     }
     if (c + 1 < chunks) fetch(c + 1);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> tensor-core reads
@@ -190,15 +191,22 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
       l0 = (double)L.v0[DAB_IDX(gl, L.rows)];
       off = kLanesAreActivations ? act_offset(gl) : gl * g.map.col_stride;
     }
+    const bool want_p11 = g.p11 != nullptr;
+    float* const crow = g.C + off;
+    // this row's counts: element (gl, j0 + j) when the lanes are activation rows, (j0 + j, gl) otherwise
+    const int64_t p0 = kLanesAreActivations ? gl * g.ldp + j0 : j0 * g.ldp + gl;
+    const int64_t pstep = kLanesAreActivations ? 1 : g.ldp;
     for (int cb = warp >> 2; cb * 32 < NT; cb += THREADS / 128) {
       uint32_t v[32];
       tmem_load_32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cb * 32), v);
       if (!valid) continue;
+      const int left = nrows - cb * 32;  // columns of this block that exist
+      const ColumnParams* const col = s_col + cb * 32;
+      const int64_t pblock = p0 + (int64_t)(cb * 32) * pstep;
 #pragma unroll
       for (int jj = 0; jj < 32; ++jj) {
-        const int j = cb * 32 + jj;
-        if (j >= nrows) break;
-        const ColumnParams cp = s_col[j];
+        if (jj >= left) break;
+        const ColumnParams cp = col[jj];
         // The four counts as doubles (small integers: every difference is exact, so these are the values
         // rescale() converts from int), then its four terms in its order: alpha gamma p11, alpha delta p10,
         // beta gamma p01, beta delta p00, with p10 the count on the weight side only.
@@ -214,9 +222,8 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) binary_gemm_mma_kernel(cons
           y = __dadd_rn(y, __dmul_rn(__dmul_rn(l0, cp.v1), pc));
         }
         y = __dadd_rn(y, __dmul_rn(__dmul_rn(cp.v0, l0), p00));
-        if (DAB_IN_BOUNDS(off + cp.off, g.c_extent)) g.C[off + cp.off] = (float)y;
-        const int64_t pidx = kLanesAreActivations ? gl * g.ldp + j0 + j : (j0 + j) * g.ldp + gl;
-        if (g.p11 && DAB_IN_BOUNDS(pidx, (g.M - 1) * g.ldp + g.N)) g.p11[pidx] = (int)v[jj];
+        if (DAB_IN_BOUNDS(off + cp.off, g.c_extent)) crow[cp.off] = (float)y;
+        if (want_p11 && DAB_IN_BOUNDS(pblock + jj * pstep, (g.M - 1) * g.ldp + g.N)) g.p11[pblock + jj * pstep] = (int)v[jj];
       }
     }
   }
@@ -254,6 +261,8 @@ cudaError_t launch_side(const GemmArgs& args, cudaStream_t stream) {
   // run best as many small CTAs (six of 128 threads per SM), wider ones as fewer CTAs of 256 threads with
   // longer stages (two per SM at the full 256 columns, where shared memory is the limit).
   if (ncap <= 64) return launch_shape<128, 1, 6, 64, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
+  if (ncap <= 128 && args.words >= 64)  // long rows: eight words per stage halve the dependent stage rounds
+    return launch_shape<256, 2, 3, 128, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
   if (ncap <= 128) return launch_shape<256, 1, 4, 128, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
   return launch_shape<256, 2, 2, MMA_NMAX, kLanesAreActivations>(args, grid, tile_cols, ncap, stream);
 }

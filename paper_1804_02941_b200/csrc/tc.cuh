@@ -27,8 +27,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 
 // Instruction descriptor of kind::i8: D format S32 (2 at bit 4), A format at bit 7 and B format at bit 10
 // (0: unsigned 8-bit, 1: signed 8-bit), both K-major (0 at bits 15 and 16), N / 8 at bit 17, M / 16 at bit 24.
-__device__ __forceinline__ uint32_t instr_desc(int nt, bool a_signed = false) {
-  return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(kLanes >> 4) << 24);
+__device__ __forceinline__ uint32_t instr_desc(int nt, bool a_signed = false, bool b_signed = false) {
+  return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | ((b_signed ? 1u : 0u) << 10) | ((uint32_t)(nt >> 3) << 17) |
+         ((uint32_t)(kLanes >> 4) << 24);
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -129,6 +130,37 @@ __device__ __forceinline__ void expand_words(uint4 q, unsigned char* dst) {
     hi.y = spread4((w[m] >> 20) & 15u);
     hi.z = spread4((w[m] >> 24) & 15u);
     hi.w = spread4(w[m] >> 28);
+    *reinterpret_cast<uint4*>(dst + (2 * m) * 128) = lo;
+    *reinterpret_cast<uint4*>(dst + (2 * m + 1) * 128) = hi;
+  }
+}
+
+// Four mask bits -> four bytes of 0 / -1 with one byte permutation: the selector's nibbles are bits s, s+4, s+8
+// and s+12 of the word shifted right by s (their lowest bit picks byte 0x00 or 0xFF of the source; the other
+// selector bits pick among copies of the same two bytes, and sign replication of 0x00 / 0xFF changes nothing).
+__device__ __forceinline__ uint32_t select4(uint32_t selector) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %1, %2;" : "=r"(d) : "r"(0xFF00FF00u), "r"(selector));
+  return d;
+}
+
+// One 16-byte piece (four mask words) of one row -> eight 16-byte K chunks of 0 / -1 bytes (signed 8-bit
+// operands: (-1) x (-1) = 1, so the integer dot product of two such rows is popc(e AND f)).  Within a word's
+// 32 bytes the bits appear in the order 0 4 8 12, 1 5 9 13, 2 6 10 14, 3 7 11 15, then the same for the upper
+// half: a permutation of the contraction index, the same on both operands, that the sum does not see.
+__device__ __forceinline__ void expand_words_signed(uint4 q, unsigned char* dst) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int m = 0; m < 4; ++m) {
+    uint4 lo, hi;
+    lo.x = select4(w[m]);
+    lo.y = select4(w[m] >> 1);
+    lo.z = select4(w[m] >> 2);
+    lo.w = select4(w[m] >> 3);
+    hi.x = select4(w[m] >> 16);
+    hi.y = select4(w[m] >> 17);
+    hi.z = select4(w[m] >> 18);
+    hi.w = select4(w[m] >> 19);
     *reinterpret_cast<uint4*>(dst + (2 * m) * 128) = lo;
     *reinterpret_cast<uint4*>(dst + (2 * m + 1) * 128) = hi;
   }
