@@ -56,17 +56,31 @@ struct PixArgs {
 // Patches of the call: the extent of pK, pgamma, pdelta and pflags (and, times ldp, of pmask).
 __device__ __forceinline__ int64_t patch_count(const PixArgs& a) { return (int64_t)a.d.N * a.Ho * a.Wo; }
 
-// Bucket grid of a tile: bucket(v) = floor(v * 2^k) + B0 for the non-zero values v, with k the largest exponent
-// that keeps every value of the tile inside the B buckets.  Multiplying by a power of two is exact, so bucket b
-// holds exactly the values in [(b - B0) 2^-k, (b - B0 + 1) 2^-k).
+// Bucket grid of a tile, one of two kinds.
+//   Both signs present: bucket(v) = floor(v * 2^k) + B0 for the non-zero values v, with k the largest exponent that
+//   keeps every value of the tile inside the B buckets.  Multiplying by a power of two is exact, so bucket b holds
+//   exactly the values in [(b - B0) 2^-k, (b - B0 + 1) 2^-k).
+//   One sign only (post-ReLU activations): buckets of equal width within each octave, 2^m per octave, over the top
+//   B / 2^m = 4 octaves of the tile's magnitudes, and one bucket from zero up to the lowest of them.  The bucket of
+//   a value is its bit pattern shifted right by 23 - m, minus a base that puts the tile's largest magnitude into
+//   the last bucket; its edges are the floats with those leading bits, so membership is exact here too.  Relative
+//   resolution is what the search needs: the best split of such rows lies among the larger values, where equal
+//   widths over the whole range would spend most buckets on values that are rare.
 struct PixQuant {
-  float scale;       // 2^k
-  double width;      // 2^-k
-  double inv_width;  // 2^k
-  int B0;            // first bucket of the positive values (0: none negative, B: none positive, B/2: both signs)
-  bool ok;           // false: magnitudes outside [2^-40, 2^40]; the tile goes to the sorting kernel
+  int shift;  // per-octave grid: 23 - m; 0: equal widths
+  int p;      // per-octave grid: the base of the shifted bit pattern; equal widths: the bits of 2^k as a float
+  int B0;     // first bucket of the positive values (0: none negative, B: none positive, B/2: both signs)
+  bool ok;    // false: magnitudes outside [2^-40, 2^40]; the tile goes to the sorting kernel
 };
 
+#ifndef DAB_PIX_OCTAVES_UPTO_BPL
+#define DAB_PIX_OCTAVES_UPTO_BPL 2  // kernels with this many buckets per lane or fewer use the per-octave grid
+#endif
+#ifndef DAB_PIX_OCTAVES_LOG2
+#define DAB_PIX_OCTAVES_LOG2 2  // the per-octave grid resolves the top 2^2 = 4 octaves of a tile's magnitudes
+#endif
+
+template <bool kOctaves>
 __device__ __forceinline__ PixQuant make_pix_quant(uint32_t kmin, uint32_t kmax, int LOG2B) {
   PixQuant q;
   const float lo = key_value(kmin), hi = key_value(kmax);
@@ -76,18 +90,49 @@ __device__ __forceinline__ PixQuant make_pix_quant(uint32_t kmin, uint32_t kmax,
   const bool mixed = lo < 0.0f && hi > 0.0f;
   const int k = (mixed ? LOG2B - 1 : LOG2B) - e - 1;
   const int kc = min(max(k, -100), 100);
-  q.scale = __uint_as_float((uint32_t)(kc + 127) << 23);
-  q.inv_width = (double)q.scale;
-  q.width = __longlong_as_double((long long)(1023 - kc) << 52);
   q.B0 = lo > 0.0f ? 0 : (hi < 0.0f ? (1 << LOG2B) : (1 << (LOG2B - 1)));
+  q.shift = 0;
+  q.p = (kc + 127) << 23;
+  if (kOctaves && !mixed) {  // 2^m buckets per octave; e >= -40 keeps the base positive
+    q.shift = 23 - (LOG2B - DAB_PIX_OCTAVES_LOG2);
+    q.p = (int)(__float_as_uint(A) >> q.shift) - ((1 << LOG2B) - 1);
+  }
   return q;
 }
 
 // (A negative value so small that the product rounds to -0.0 still belongs below zero.)
+template <bool kOctaves>
 __device__ __forceinline__ int pix_bucket(float v, const PixQuant& q, int B) {
-  int f = __float2int_rd(v * q.scale);
+  if (kOctaves && q.shift) {  // one sign only: magnitudes ascend with the bucket for positive tiles, descend for negative ones
+    const int i = min(max((int)((__float_as_uint(v) & 0x7FFFFFFFu) >> q.shift) - q.p, 0), B - 1);
+    return q.B0 ? B - 1 - i : i;
+  }
+  int f = __float2int_rd(v * __int_as_float(q.p));
   if (v < 0.0f) f = min(f, -1);
   return min(max(f + q.B0, 0), B - 1);
+}
+
+// Values bucket b can hold, [vlo, vhi), and the reciprocal of its width (exact for every bucket but the one next
+// to zero of the per-octave grid, where it is good to 2 ulp of fp32: it only places the corners of a bound that
+// is compared with a margin of 2e-5).
+template <bool kOctaves>
+__device__ __forceinline__ void pix_bucket_range(const PixQuant& q, int b, int B, double& vlo, double& vhi,
+                                                 double& inv_width) {
+  if (kOctaves && q.shift) {
+    const int i = q.B0 ? B - 1 - b : b;
+    const float lo = i ? __uint_as_float((uint32_t)(i + q.p) << q.shift) : 0.0f;
+    const float hi = __uint_as_float((uint32_t)(i + 1 + q.p) << q.shift);
+    vlo = q.B0 ? -(double)hi : (double)lo;
+    vhi = q.B0 ? -(double)lo : (double)hi;
+    // hi - lo = 2^(exponent of lo - m) with m = 23 - shift: its reciprocal by exponent arithmetic; next to zero 1 / hi
+    const int biased = (int)((uint32_t)(i + q.p) >> (23 - q.shift));  // exponent field of lo
+    inv_width = i ? (double)__int_as_float((254 + (23 - q.shift) - biased) << 23) : (double)__fdividef(1.0f, hi);
+    return;
+  }
+  const double width = (double)__int_as_float((254 << 23) - q.p);  // q.p holds the bits of 2^k: 2^-k, exact
+  vlo = (double)(b - q.B0) * width;
+  vhi = vlo + width;
+  inv_width = (double)__int_as_float(q.p);
 }
 
 // Objective in fp32 from fp64 coordinates: every input is rounded once (relative 2^-24), both terms are
@@ -152,6 +197,7 @@ template <int WARPS, int MINB, int BPL, int KHW, typename ListT, bool kTable>
 __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_kernel(const PixArgs a) {
   constexpr int THREADS = WARPS * 32;
   constexpr int B = 32 * BPL;
+  constexpr bool kOctaves = BPL <= DAB_PIX_OCTAVES_UPTO_BPL;  // single-signed tiles take the per-octave grid
   constexpr int LOG2B = BPL == 1 ? 5 : BPL == 2 ? 6 : BPL == 4 ? 7 : 8;
   constexpr int SS = B + 1;  // table row stride: odd, so that one thread per pixel walks its row without conflicts
   constexpr int KMAX = KHW ? KHW : 1;
@@ -256,7 +302,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     __syncthreads();
     const uint32_t tkmin = s_kmin, tkmax = s_kmax;
     const bool any_nonzero = tkmin <= tkmax;
-    PixQuant qz = make_pix_quant(any_nonzero ? tkmin : kZeroKey + 1u, any_nonzero ? tkmax : kZeroKey + 1u, LOG2B);
+    PixQuant qz = make_pix_quant<kOctaves>(any_nonzero ? tkmin : kZeroKey + 1u, any_nonzero ? tkmax : kZeroKey + 1u, LOG2B);
     if (any_nonzero && (key_range_nonfinite(tkmin, tkmax) || !qz.ok)) {
       // every patch of the tile is left to the sorting kernel
       for (int p = threadIdx.x; p < npatch; p += THREADS) {
@@ -271,7 +317,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
       for (int c = warp; c < C; c += WARPS) {
         const float v = tile[c * chw + p];
         if (v != 0.0f) {
-          const int slot = p * SS + pix_bucket(v, qz, B);
+          const int slot = p * SS + pix_bucket<kOctaves>(v, qz, B);
           atomicAdd(&cntc[slot], 1);
           atomicAdd(&sumc[slot], (double)v);
         }
@@ -299,7 +345,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
       for (int c = warp; c < C; c += WARPS) {
         const float v = tile[c * chw + p];
         if (v != 0.0f) {
-          const int pos = atomicAdd(&cntc[p * SS + pix_bucket(v, qz, B)], 1);
+          const int pos = atomicAdd(&cntc[p * SS + pix_bucket<kOctaves>(v, qz, B)], 1);
           list[p * C + pos] = (ListT)c;
         }
       }
@@ -400,9 +446,10 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
           if (c >= 2) {
             // value bounds of the bucket and the two inner corners of the region (s, P) can visit inside it
             const int s0 = pc[j] + (b >= qz.B0 ? z : 0);
-            const double vlo = (double)(b - qz.B0) * qz.width, vhi = vlo + qz.width;
+            double vlo, vhi, inv_width;
+            pix_bucket_range<kOctaves>(qz, b, B, vlo, vhi, inv_width);
             const double cd = (double)c, S = cs[j] - ps[j];
-            double jl = (cd * vhi - S) * qz.inv_width;
+            double jl = (cd * vhi - S) * inv_width;
             jl = fmin(fmax(jl, 0.0), cd);
             const double ju = cd - jl;
             dk = fmaxf(objective_bound((double)s0 + jl, ps[j] + jl * vlo, T, nd),
@@ -467,10 +514,12 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
                 if (lane >= o) incl += t;
               }
               const int excl = incl - my_len;
-              // (no one-key-per-lane variant for the smallest hulls: the extra code costs more in instruction fetches
-              // than its shorter network saves)
+              // (a one-key-per-lane search pays only where hulls of up to 32 values are the rule, i.e. under the
+              // per-octave grid; elsewhere its extra code costs more in instruction fetches than it saves)
               if (__shfl_sync(0xFFFFFFFFu, incl, KMAX - 1) != m_sub) {
                 retry = true;  // cannot happen; never trust a mismatch
+              } else if (kOctaves && m_sub <= 32) {  // the usual case under the per-octave grid
+                res = pix_gather_sort_select<1, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
               } else if (m_sub <= 64) {
                 res = pix_gather_sort_select<2, kTable>(tile, list, C, chw, excl, my_st, my_pq, KMAX, m_sub, z_in, a.n, lane, rcp, base);
               } else if (m_sub <= 128) {
