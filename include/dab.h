@@ -371,13 +371,14 @@ dab_contraction dab_get_contraction(void);
  *                      buckets whose bound reaches the best edge value are searched exactly.  Work per pixel is
  *                      shared by the up to kh*kw patches that contain it.  Patches it cannot settle (a hull of more
  *                      than 1024 values, a constant row without zeros, magnitudes outside 2^-40..2^40, a NaN or an
- *                      infinity in the tile) are sorted in full by a second kernel;
+ *                      infinity in the tile) are sorted in full by a last kernel.  Rows of 1024 values and more
+ *                      run as two such kernels: the first, with half the buckets, codes the tiles whose non-zero
+ *                      values have one sign; the second codes the tiles with both signs;
  *   DAB_PATCHES_HIST   rows and patches of 257..8192 values, one warp each: a histogram of the row's own values
  *                      quantised to 24 bits of its range, the same bound per bucket with a margin for the
  *                      quantisation, exact search of what survives; rows it cannot settle fall to the sorting kernel;
  *   DAB_PATCHES_AUTO   (default) patches: DAB_PATCHES_PIXEL wherever a patch spans several pixels and the layer has
- *                      at least 1024 patches (except strided windows over more than 128 channels, which overlap too
- *                      little); otherwise per tile of the input the sorting kernels for tiles with few non-zero values
+ *                      at least 1024 patches; otherwise per tile of the input the sorting kernels for tiles with few non-zero values
  *                      and DAB_PATCHES_HIST for the others.  Rows of a matrix: DAB_PATCHES_HIST from 2048 rows on,
  *                      DAB_PATCHES_SORT below.
  * Process-wide, read once at the start of each call.

@@ -623,9 +623,8 @@ cudaError_t launch_binarize_patches(const dab_conv_desc& d, int32_t Ho, int32_t 
   cudaError_t e;
   // The pixel-histogram coder shares work between overlapping patches: it is the default wherever a patch spans
   // several pixels and the layer has enough patches to fill the device with its tiles (measured: from about a
-  // thousand patches; strided windows over many channels overlap too little to gain).
-  const bool pixel_default = d.kh * d.kw >= 4 && (int64_t)d.N * Ho * Wo >= 1024 &&
-                             !(d.stride_h * d.stride_w >= 4 && d.C > 128);
+  // thousand patches).
+  const bool pixel_default = d.kh * d.kw >= 4 && (int64_t)d.N * Ho * Wo >= 1024;
   if (mode == 3 || (mode == 0 && pixel_default)) {
     bool applicable = false;
     e = launch_binarize_patches_pixhist(d, Ho, Wo, x, pK, pgamma, pdelta, pmask, ldp, pflags, stream, &applicable);

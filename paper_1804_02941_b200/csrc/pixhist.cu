@@ -51,6 +51,8 @@ struct PixArgs {
   uint32_t* pflags;  // may be null
   uint32_t* pmask;
   int32_t ldp;
+  int32_t defer_mixed;  // leave tiles that hold both signs to the next kernel of the call (marks all their patches)
+  int32_t marked_only;  // code only the tiles whose first patch carries the mark of the kernel before
 };
 
 // Patches of the call: the extent of pK, pgamma, pdelta and pflags (and, times ldp, of pmask).
@@ -73,8 +75,13 @@ struct PixQuant {
   bool ok;    // false: magnitudes outside [2^-40, 2^40]; the tile goes to the sorting kernel
 };
 
+#ifndef DAB_PIX_N1
+#define DAB_PIX_N1 1024  // rows shorter than this: 32 buckets, tiles of both signs coded in place
+#define DAB_PIX_N2 2048  // ... than this: 32 buckets, then 64 for the tiles with both signs
+#define DAB_PIX_N4 4096  // ... than this: 64, then 128; longer rows: 128, then 256
+#endif
 #ifndef DAB_PIX_OCTAVES_UPTO_BPL
-#define DAB_PIX_OCTAVES_UPTO_BPL 2  // kernels with this many buckets per lane or fewer use the per-octave grid
+#define DAB_PIX_OCTAVES_UPTO_BPL 4  // kernels with this many buckets per lane or fewer use the per-octave grid
 #endif
 #ifndef DAB_PIX_OCTAVES_LOG2
 #define DAB_PIX_OCTAVES_LOG2 2  // the per-octave grid resolves the top 2^2 = 4 octaves of a tile's magnitudes
@@ -214,6 +221,18 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
   ListT* list = reinterpret_cast<ListT*>(off + (KHW ? 0 : ((a.n + 1) & ~1)));  // [pix][C] channels by bucket
 
   __shared__ uint32_t s_kmin, s_kmax;
+  if (a.marked_only) {
+    // the second kernel of a call usually has nothing to do: every thread looks at the first patch of another of
+    // the CTA's tiles, and the CTA leaves before any set-up unless one of them carries the mark
+    const int64_t per_img = (int64_t)a.tiles_h * a.tiles_w, tiles = per_img * a.d.N;
+    int any = 0;
+    for (int64_t t = blockIdx.x + (int64_t)threadIdx.x * gridDim.x; t < tiles; t += (int64_t)THREADS * gridDim.x) {
+      const int img = (int)(t / per_img), trem = (int)(t % per_img);
+      const int64_t first = ((int64_t)img * a.Ho + (trem / a.tiles_w) * a.TH) * a.Wo + (trem % a.tiles_w) * a.TW;
+      any |= a.pK[DAB_IDX(first, patch_count(a))] == kRowMark;
+    }
+    if (!__syncthreads_or(any)) return;
+  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int C = a.d.C, pixn = a.pix, chw = a.ch_words, khw = a.d.kh * a.d.kw;
   uint32_t* scratch = scratch_all + warp * kHullCap;
@@ -249,6 +268,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     const int th = min(a.TH, a.Ho - ho0), tw = min(a.TW, a.Wo - wo0);
     const int npatch = th * tw;
     const int64_t tile_base = ((int64_t)img * a.Ho + ho0) * a.Wo + wo0;  // index of the tile's first patch
+    if (a.marked_only && a.pK[DAB_IDX(tile_base, patch_count(a))] != kRowMark) continue;  // the same for every thread
     __syncthreads();  // the previous tile is no longer read
     if (threadIdx.x == 0) { s_kmin = kPadKey; s_kmax = 0u; }
     for (int i = threadIdx.x; i < pixn * SS; i += THREADS) { cntc[i] = 0; sumc[i] = 0.0; }
@@ -303,8 +323,9 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     const uint32_t tkmin = s_kmin, tkmax = s_kmax;
     const bool any_nonzero = tkmin <= tkmax;
     PixQuant qz = make_pix_quant<kOctaves>(any_nonzero ? tkmin : kZeroKey + 1u, any_nonzero ? tkmax : kZeroKey + 1u, LOG2B);
-    if (any_nonzero && (key_range_nonfinite(tkmin, tkmax) || !qz.ok)) {
-      // every patch of the tile is left to the sorting kernel
+    const bool both_signs = any_nonzero && key_value(tkmin) < 0.0f && key_value(tkmax) > 0.0f;
+    if (any_nonzero && (key_range_nonfinite(tkmin, tkmax) || !qz.ok || (a.defer_mixed && both_signs))) {
+      // every patch of the tile is left to the next kernel of the call
       for (int p = threadIdx.x; p < npatch; p += THREADS) {
         const int64_t pi = tile_base + (int64_t)(p / tw) * a.Wo + p % tw;
         if (DAB_IN_BOUNDS(pi, patch_count(a))) a.pK[pi] = kRowMark;
@@ -752,7 +773,7 @@ cudaError_t launch_pix_minb(PixArgs& a, size_t smem, cudaStream_t stream) {
 }
 
 #ifndef DAB_PIX_WIDE_FROM_BPL
-#define DAB_PIX_WIDE_FROM_BPL 4   // buckets per lane from which a CTA has 16 warps instead of 8
+#define DAB_PIX_WIDE_FROM_BPL 2   // buckets per lane from which a CTA has 16 warps instead of 8
 #endif
 #ifndef DAB_PIX_WARPS
 #define DAB_PIX_WARPS 8
@@ -768,7 +789,7 @@ cudaError_t launch_pix(PixArgs& a, cudaStream_t stream, bool* applicable) {
   // rows of 2048 values and more leave room for one to three CTAs per SM only (tables, values and lists of a pixel
   // take 3 to 6 KB): their CTAs get twice the warps
   constexpr int W = BPL >= DAB_PIX_WIDE_FROM_BPL ? 2 * DAB_PIX_WARPS : DAB_PIX_WARPS;
-  constexpr int kMostCtas = BPL <= DAB_PIX_FOUR_CTAS_UPTO_BPL ? 4 : 3;
+  constexpr int kMostCtas = (W == DAB_PIX_WARPS && BPL <= DAB_PIX_FOUR_CTAS_UPTO_BPL) ? 4 : 3;
   PixArgs cand[4] = {a, a, a, a};
   size_t smem[4] = {0, 0, 0, 0};
   double cost[4] = {0, 0, 0, 0};
@@ -799,7 +820,7 @@ cudaError_t launch_pix_for(PixArgs& a, cudaStream_t stream, bool* applicable) {
   constexpr bool kTable = BPL <= 2;
   if (a.d.kh == 3 && a.d.kw == 3) {
     if (a.d.C <= 256) return launch_pix<BPL, 9, uint8_t, kTable>(a, stream, applicable);
-    if constexpr (BPL >= 4) return launch_pix<BPL, 9, uint16_t, kTable>(a, stream, applicable);
+    if constexpr (BPL >= 2) return launch_pix<BPL, 9, uint16_t, kTable>(a, stream, applicable);
   }
   return launch_pix<BPL, 0, uint16_t, kTable>(a, stream, applicable);
 }
@@ -831,15 +852,33 @@ cudaError_t launch_binarize_patches_pixhist(const dab_conv_desc& d, int32_t Ho, 
   *applicable = false;
   if (a.n <= 256 || a.n > 8192 || d.kh * d.kw > 64) return cudaSuccess;
   cudaError_t e;
-  // buckets by patch length: about n / 18, so that the two to four buckets that survive hold a few dozen values
-  // (measured against half and twice as many: fewer buckets leave hulls that are slow on inputs without zeros, more
-  // cost their tables in shared memory and their bounds per patch more than the smaller hulls save)
-  if (a.n < 1024) e = launch_pix_for<1>(a, stream, applicable);
-  else if (a.n < 2048) e = launch_pix_for<2>(a, stream, applicable);
-  else if (a.n < 4096) e = launch_pix_for<4>(a, stream, applicable);
-  else e = launch_pix_for<8>(a, stream, applicable);
+  // Buckets by patch length.  Tiles of one sign (post-ReLU activations) take the per-octave grid, under which 32
+  // buckets leave a hull of about 17 values of a row of 576 and of about 36 of a row of 1152; the first kernel is
+  // sized for them.  A tile with both signs needs the equal-width grid with twice the buckets: rows of 1024 values
+  // and more leave such tiles (all their patches marked) to a second kernel with twice the buckets per lane, which
+  // looks at the first patch of every tile and codes the marked tiles only.
+  a.defer_mixed = a.n >= DAB_PIX_N1 ? 1 : 0;
+  a.marked_only = 0;
+  PixArgs second = a;
+  second.defer_mixed = 0;
+  second.marked_only = 1;
+  bool second_fits = false;
+  if (a.n < DAB_PIX_N1) {
+    e = launch_pix_for<1>(a, stream, applicable);
+  } else if (a.n < DAB_PIX_N2) {
+    e = launch_pix_for<1>(a, stream, applicable);
+    if (e == cudaSuccess && *applicable) e = launch_pix_for<2>(second, stream, &second_fits);
+  } else if (a.n < DAB_PIX_N4) {
+    e = launch_pix_for<2>(a, stream, applicable);
+    if (e == cudaSuccess && *applicable) e = launch_pix_for<4>(second, stream, &second_fits);
+  } else {
+    e = launch_pix_for<4>(a, stream, applicable);
+    if (e == cudaSuccess && *applicable) e = launch_pix_for<8>(second, stream, &second_fits);
+  }
+  // (a second kernel that fits no tile launches nothing: the marked tiles then go to the sorting kernel below)
   if (e != cudaSuccess || !*applicable) return e;
   if (a.n <= 2048) return launch_fixup<8>(a, stream);
+  if (a.n <= 4096) return launch_fixup<16>(a, stream);
   return launch_fixup<32>(a, stream);
 }
 
