@@ -651,10 +651,11 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
 // ---------------------------------------------------------------------------------------------------------
 // The kernel that follows on the stream: patches marked K = kRowMark are coded by the full sort of rowcode.cuh,
 // one CTA (a group of 8 warps) per marked patch, values read straight from global memory.  Every CTA looks at a
-// run of 256 patch slots at a time and queues the marked ones.
+// run of `run` (32 to 256) patch slots at a time and queues the marked ones; short runs spread the marked patches
+// of a small layer over all SMs.
 // ---------------------------------------------------------------------------------------------------------
 template <int R>
-__global__ void __launch_bounds__(kFixThreads) binarize_patches_fixup_kernel(const PixArgs a, int scratch_words) {
+__global__ void __launch_bounds__(kFixThreads) binarize_patches_fixup_kernel(const PixArgs a, int scratch_words, int run) {
   constexpr int W = kFixWarps;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   GroupShared* gs = reinterpret_cast<GroupShared*>(smem_raw);
@@ -664,11 +665,11 @@ __global__ void __launch_bounds__(kFixThreads) binarize_patches_fixup_kernel(con
   const int tig = threadIdx.x;
   const int64_t total = (int64_t)a.d.N * a.Ho * a.Wo;
   const int khw = a.d.kh * a.d.kw;
-  for (int64_t chunk = (int64_t)blockIdx.x * kFixThreads; chunk < total; chunk += (int64_t)gridDim.x * kFixThreads) {
+  for (int64_t chunk = (int64_t)blockIdx.x * run; chunk < total; chunk += (int64_t)gridDim.x * run) {
     __syncthreads();
     if (tig == 0) qn = 0;
     __syncthreads();
-    if (chunk + tig < total && a.pK[DAB_IDX(chunk + tig, total)] == kRowMark) queue[atomicAdd(&qn, 1)] = tig;
+    if (tig < run && chunk + tig < total && a.pK[DAB_IDX(chunk + tig, total)] == kRowMark) queue[atomicAdd(&qn, 1)] = tig;
     __syncthreads();
     const int count = qn;
     for (int qi = 0; qi < count; ++qi) {
@@ -833,9 +834,11 @@ cudaError_t launch_fixup(const PixArgs& a, cudaStream_t stream) {
   cudaError_t e = ensure_dynamic_smem(kern, smem);
   if (e != cudaSuccess) return e;
   const int64_t total = (int64_t)a.d.N * a.Ho * a.Wo;
-  int64_t blocks = (total + kFixThreads - 1) / kFixThreads;
+  int run = kFixThreads;  // patch slots a CTA scans at a time: fewer for small layers, so that every SM gets some
+  while (run > 32 && (total + run - 1) / run < 4 * (int64_t)sm_count()) run >>= 1;
+  int64_t blocks = (total + run - 1) / run;
   if (blocks > sm_count() * 4) blocks = sm_count() * 4;
-  kern<<<(unsigned)blocks, kFixThreads, smem, stream>>>(a, sw);
+  kern<<<(unsigned)blocks, kFixThreads, smem, stream>>>(a, sw, run);
   return cudaGetLastError();
 }
 

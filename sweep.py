@@ -154,7 +154,56 @@ def network_point(name, build, batch):
          binarized_layers=sum(l["kind"] == "conv_binary" for l in layers))
 
 
+def table(path):
+    """Markdown summary of the JSON lines an earlier run printed (python sweep.py ... > lines; python sweep.py --table lines)."""
+    recs = [json.loads(l) for l in open(path) if l.lstrip().startswith("{")]
+    peaks = next((r["peaks"] for r in recs if "peaks" in r), {})
+    int8_peak = None
+    try:
+        int8_peak = 2.0 * json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"]
+    except Exception:
+        pass
+    print("| config | layer / point | stage | ms | rate | fraction |")
+    print("|---|---|---|---|---|---|")
+    nets = []
+    for r in recs:
+        st = r.get("stage")
+        if st is None:
+            continue
+        if st == "network_forward":
+            nets.append(r)
+            continue
+        if "layer" in r:
+            where = "%s%s (n=%d, %d patches, %d filters)" % (r["layer"], " dense" if r.get("inputs", "").startswith("dense") else "",
+                                                             r["n"], r["patches"], r["filters"])
+        elif st == "pack":
+            where = "%d x %d bytes" % (r["rows"], r["n"])
+        else:
+            where = "M=N=%d, n=%d" % (r["M"], r["n"])
+        if "gbs" in r:
+            rate, frac = "%.1f GB/s" % r["gbs"], "hbm %.4f" % r["hbm_frac"]
+        elif "tmacs" in r:
+            rate, frac = "%.1f TMAC/s" % r["tmacs"], "int8 %.3f" % r["int8_frac"]
+        else:
+            rate = "%.1f TOPS-eq" % r["tops_equiv"]
+            frac = ""
+            if "alu_frac" in r:
+                frac = "alu %.2f" % r["alu_frac"] + (", int8 %.3f" % (r["tops_equiv"] / int8_peak) if int8_peak else "")
+        name = {"conv_total": "patches + contract", "binarize": "binarize rows"}.get(st, st)
+        print("| %s | %s | %s | %.4f | %s | %s |" % (r.get("config", "pack"), where, name, r["ms"], rate, frac))
+    if nets:
+        print("\n| network | batch | layers (binarized) | ms | images/s |\n|---|---|---|---|---|")
+        for r in nets:
+            print("| %s | %d | %d (%d) | %.3f | %.0f |" % (r["network"], r["batch"], r["layers"], r["binarized_layers"], r["ms"], r["images_per_s"]))
+    if peaks:
+        print("\nPeaks used: HBM %.1f GB/s (%s); population-count bound %.1f TOPS-equiv (%s)%s." % (
+            peaks["hbm_gbs"], peaks["source"], peaks["contraction_tops_equiv"], peaks["contraction_peak"],
+            "; int8 tensor peak %.0f TOPS" % int8_peak if int8_peak else ""))
+
+
 def main():
+    if len(sys.argv) == 3 and sys.argv[1] == "--table":
+        return table(sys.argv[2])
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--batch5", type=int, default=256)
