@@ -120,8 +120,7 @@ __device__ __forceinline__ int pix_bucket(float v, const PixQuant& q, int B) {
 }
 
 // Values bucket b can hold, [vlo, vhi), and the reciprocal of its width (exact for every bucket but the one next
-// to zero of the per-octave grid, where it is good to 2 ulp of fp32: it only places the corners of a bound that
-// is compared with a margin of 2e-5).
+// to zero of the per-octave grid, where it is good to 2e-14 relative).
 template <bool kOctaves>
 __device__ __forceinline__ void pix_bucket_range(const PixQuant& q, int b, int B, double& vlo, double& vhi,
                                                  double& inv_width) {
@@ -133,7 +132,9 @@ __device__ __forceinline__ void pix_bucket_range(const PixQuant& q, int b, int B
     vhi = q.B0 ? -(double)lo : (double)hi;
     // hi - lo = 2^(exponent of lo - m) with m = 23 - shift: its reciprocal by exponent arithmetic; next to zero 1 / hi
     const int biased = (int)((uint32_t)(i + q.p) >> (23 - q.shift));  // exponent field of lo
-    inv_width = i ? (double)__int_as_float((254 + (23 - q.shift) - biased) << 23) : (double)__fdividef(1.0f, hi);
+    const double r = i ? (double)__int_as_float((254 + (23 - q.shift) - biased) << 23) : (double)__fdividef(1.0f, hi);
+    // one Newton step: leaves the exact reciprocals as they are and takes 1 / hi from 2 ulp of fp32 to 2e-14 relative
+    inv_width = __dmul_rn(r, __dsub_rn(2.0, __dmul_rn(vhi - vlo, r)));
     return;
   }
   const double width = (double)__int_as_float((254 << 23) - q.p);  // q.p holds the bits of 2^k: 2^-k, exact
