@@ -75,6 +75,10 @@ struct PixQuant {
   bool ok;    // false: magnitudes outside [2^-40, 2^40]; the tile goes to the sorting kernel
 };
 
+#ifndef DAB_PIX_COST_PATCH
+#define DAB_PIX_COST_PATCH 5000.0  // cost model of the tile choice: cycles per patch, ...
+#define DAB_PIX_COST_VALUE 5.0     // ... plus this per value of the patch (a staged value of the tile costs 4.6)
+#endif
 #ifndef DAB_PIX_N1
 #define DAB_PIX_N1 1024  // rows shorter than this: 32 buckets, tiles of both signs coded in place
 #define DAB_PIX_N2 2048  // ... than this: 32 buckets, then 64 for the tiles with both signs
@@ -736,7 +740,7 @@ bool choose_pix_tile(PixArgs* a, size_t budget, int ctas_per_sm, size_t* smem_ou
   double best_cost = 0.0;
   int best_th = 0, best_tw = 0;
   size_t best_smem = 0;
-  const double per_patch = 5000.0 + 5.0 * a->n;
+  const double per_patch = DAB_PIX_COST_PATCH + DAB_PIX_COST_VALUE * a->n;
   const int sms = sm_count();
   for (int th = 8; th >= 1; --th) {
     for (int tw = 8; tw >= 1; --tw) {
