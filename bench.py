@@ -433,7 +433,7 @@ def run_dab(args):
                              "popc_bound_source": "the integer-pipe bound of the population-count kernel (16 popc/clk/SM x "
                                                   "1.5 words per popc x SMs x max clock x 64): what the same contraction "
                                                   "could reach without tensor cores",
-                             "note": "kind::i8 on 0/1 bytes; the kernel's time goes to expanding mask words to bytes, the fp64 "
+                             "note": "kind::i8 on masks expanded to bytes 0 / -1; the kernel's time goes to expanding mask words to bytes, the fp64 "
                                      "rescale of every count and the output store, not to the tensor pipe", **common}
     else:
         roofline_contract = {"kernel": "binary_gemm_kernel", "bound": "alu", "peak": popc_peak_derived,
