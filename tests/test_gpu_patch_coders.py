@@ -121,6 +121,28 @@ def test_mixed_density_batches_split_between_the_coders(dab):
         assert torch.equal(s, au)
 
 
+@pytest.mark.parametrize("C", [128, 256, 512])
+def test_pixel_coder_regions_of_one_sign_and_of_both_in_one_image(dab, C):
+    # rows of 1024 values and more: tiles of one sign (either one) are coded by the first launch, tiles with both signs
+    # by the second; the regions meet inside tiles as well
+    x = dab_synth.relu_activations((2, C, 16, 16), 0.6, stream=1200 + C).astype(np.float32)
+    x[:, :, :, 9:] = dab_synth.normal((2, C, 16, 7), 1.0, stream=1300 + C)
+    x[1, :, :7, :9] = -x[1, :, :7, :9]
+    xd = to_dev(x)
+    a = _code(dab, xd, C, 3, 3, (1, 1), (1, 1), dab.PATCHES_SORT)
+    px = _code(dab, xd, C, 3, 3, (1, 1), (1, 1), dab.PATCHES_PIXEL)
+    for s, pp in zip(a, px):
+        assert torch.equal(s, pp)
+    n = C * 9
+    rows = oracle.im2col(x, 3, 3, (1, 1), (1, 1))
+    sel = np.unique((dab_synth.uniform01(97, C, 0, 96) * len(rows)).astype(np.int64))
+    ref = oracle.binarize(rows[sel])
+    strict = ~((ref.gap > 0) & (ref.gap < NEAR_TIE))
+    t = torch.from_numpy(sel).to(xd.device)
+    assert np.array_equal(px[0][t].cpu().numpy()[strict], ref.K[strict])
+    assert np.array_equal(unpack(words(px[3][t]), n)[strict], ref.e[strict])
+
+
 @pytest.mark.parametrize("n", [257, 300, 575, 576, 577, 1024, 1152, 1600, 2304, 4096, 4608, 8192])
 @pytest.mark.parametrize("kind", ["normal", "relu", "laplace", "ints", "cluster", "negative"])
 def test_rows_of_a_matrix_through_both_coders(dab, n, kind):
