@@ -45,7 +45,9 @@ def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False
         return LIB
     os.makedirs(OBJDIR, exist_ok=True)
     nvcc = _nvcc()
-    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DDAB_DEBUG_BOUNDS"] if debug_bounds else [])
+    # the checking build is compiled with -split-compile 0 (the kernels of a translation unit optimised in parallel
+    # on all cores: a third of the time); the ordinary build is not: its patch coder measured 6 % slower that way
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DDAB_DEBUG_BOUNDS", "-split-compile", "0"] if debug_bounds else [])
 
     def compile_one(src):
         obj = os.path.join(OBJDIR, os.path.basename(src)[:-3] + ".o")
