@@ -235,9 +235,7 @@ def patch_launches(L, coder):
         return 1
     pixel = n <= 8192 and L.kh * L.kw >= 4 and L.patches >= 1024
     if coder == "pixel" or (coder == "auto" and pixel):
-        # pixel-histogram coder (from 1024 values on a second one for tiles with both signs), then the kernel that
-        # sorts the patches they marked
-        return 2 if n < 1024 else 3
+        return 2                      # pixel-histogram coder, then the kernel that sorts the patches it marked
     if coder == "auto":
         return 3                      # sort-based coder, histogram coder on the dense tiles, group kernel on the rest
     if coder == "hist":
@@ -398,8 +396,8 @@ def run_dab(args):
     patch_bytes = sum(4 * L.N * L.C * L.H * L.W + L.patches * (4 * dab.dab_words_per_row(L.n) + 12) for L in layers)
     binarize_gbs = patch_bytes * args.steps / (k_ms["binarize_patches"] * 1e-3) / 1e9
     traffic = measured_patch_coder_traffic([L.name for L in layers], args.batch, args.dense) if args.patch_coder == "auto" else None
-    roofline = {"kernel": "binarize_patches_pixhist_kernel (+ its second launch for tiles with both signs and "
-                          "binarize_patches_fixup_kernel, which end at once on this workload)", "bound": "hbm", "achieved": binarize_gbs,
+    roofline = {"kernel": "binarize_patches_pixhist_kernel (+ binarize_patches_fixup_kernel, which finds nothing marked on "
+                          "this workload)", "bound": "hbm", "achieved": binarize_gbs,
                 "peak": hbm_peak, "unit": "GB/s", "frac": binarize_gbs / hbm_peak, "traffic": traffic,
                 "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum per layer launch, average over the layers, from "
                                 "profiles/patch_coder_dram_traffic.json; null when the coder's sources have changed since "

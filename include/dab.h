@@ -371,9 +371,7 @@ dab_contraction dab_get_contraction(void);
  *                      buckets whose bound reaches the best edge value are searched exactly.  Work per pixel is
  *                      shared by the up to kh*kw patches that contain it.  Patches it cannot settle (a hull of more
  *                      than 1024 values, a constant row without zeros, magnitudes outside 2^-40..2^40, a NaN or an
- *                      infinity in the tile) are sorted in full by a last kernel.  Rows of 1024 values and more
- *                      run as two such kernels: the first, with half the buckets, codes the tiles whose non-zero
- *                      values have one sign; the second codes the tiles with both signs;
+ *                      infinity in the tile) are sorted in full by a second kernel;
  *   DAB_PATCHES_HIST   rows and patches of 257..8192 values, one warp each: a histogram of the row's own values
  *                      quantised to 24 bits of its range, the same bound per bucket with a margin for the
  *                      quantisation, exact search of what survives; rows it cannot settle fall to the sorting kernel;

@@ -51,23 +51,24 @@ struct PixArgs {
   uint32_t* pflags;  // may be null
   uint32_t* pmask;
   int32_t ldp;
-  int32_t defer_mixed;  // leave tiles that hold both signs to the next kernel of the call (marks all their patches)
-  int32_t marked_only;  // code only the tiles whose first patch carries the mark of the kernel before
 };
 
 // Patches of the call: the extent of pK, pgamma, pdelta and pflags (and, times ldp, of pmask).
 __device__ __forceinline__ int64_t patch_count(const PixArgs& a) { return (int64_t)a.d.N * a.Ho * a.Wo; }
 
-// Bucket grid of a tile, one of two kinds.
-//   Both signs present: bucket(v) = floor(v * 2^k) + B0 for the non-zero values v, with k the largest exponent that
-//   keeps every value of the tile inside the B buckets.  Multiplying by a power of two is exact, so bucket b holds
-//   exactly the values in [(b - B0) 2^-k, (b - B0 + 1) 2^-k).
-//   One sign only (post-ReLU activations): buckets of equal width within each octave, 2^m per octave, over the top
-//   B / 2^m = 4 octaves of the tile's magnitudes, and one bucket from zero up to the lowest of them.  The bucket of
-//   a value is its bit pattern shifted right by 23 - m, minus a base that puts the tile's largest magnitude into
-//   the last bucket; its edges are the floats with those leading bits, so membership is exact here too.  Relative
-//   resolution is what the search needs: the best split of such rows lies among the larger values, where equal
-//   widths over the whole range would spend most buckets on values that are rare.
+// Bucket grid of a tile: buckets of equal width within each octave of magnitude, 2^m per octave.  The bucket of a
+// value is the bit pattern of its magnitude shifted right by 23 - m, minus a base that puts the tile's largest
+// magnitude into the last bucket of its side; everything below the resolved octaves shares the bucket next to zero.
+// The edges are the floats with those leading bits, so membership is exact.
+//   One sign only (post-ReLU activations): all B buckets over the top B / 2^m = 4 octaves.  The best split of such
+//   rows lies among the larger values.
+//   Both signs: B/2 buckets on either side of zero over the top 8 octaves.  Such rows often split near zero, where
+//   this grid is finest in absolute terms, and a heavy tail costs it one bucket per half octave instead of
+//   stretching every bucket.
+// Relative resolution is what the search needs: buckets of one width over the whole range spend most of them where
+// values are rare, and one outlier in the tile widens them all.  (Kernels compiled without kOctaves use that
+// equal-width grid, bucket(v) = floor(v * 2^k) + B0 with k the largest exponent that fits the range; none is by
+// default.)
 struct PixQuant {
   int shift;  // per-octave grid: 23 - m; 0: equal widths
   int p;      // per-octave grid: the base of the shifted bit pattern; equal widths: the bits of 2^k as a float
@@ -79,16 +80,18 @@ struct PixQuant {
 #define DAB_PIX_COST_PATCH 5000.0  // cost model of the tile choice: cycles per patch, ...
 #define DAB_PIX_COST_VALUE 5.0     // ... plus this per value of the patch (a staged value of the tile costs 4.6)
 #endif
-#ifndef DAB_PIX_N1
-#define DAB_PIX_N1 1024  // rows shorter than this: 32 buckets, tiles of both signs coded in place
-#define DAB_PIX_N2 2048  // ... than this: 32 buckets, then 64 for the tiles with both signs
-#define DAB_PIX_N4 4096  // ... than this: 64, then 128; longer rows: 128, then 256
+#ifndef DAB_PIX_N2
+#define DAB_PIX_N2 2048  // rows shorter than this take 32 buckets, ...
+#define DAB_PIX_N4 4096  // ... than this 64, longer ones 128
 #endif
 #ifndef DAB_PIX_OCTAVES_UPTO_BPL
-#define DAB_PIX_OCTAVES_UPTO_BPL 4  // kernels with this many buckets per lane or fewer use the per-octave grid
+#define DAB_PIX_OCTAVES_UPTO_BPL 8  // kernels with this many buckets per lane or fewer use the per-octave grid
 #endif
 #ifndef DAB_PIX_OCTAVES_LOG2
-#define DAB_PIX_OCTAVES_LOG2 2  // the per-octave grid resolves the top 2^2 = 4 octaves of a tile's magnitudes
+#define DAB_PIX_OCTAVES_LOG2 2        // the per-octave grid resolves the top 2^2 = 4 octaves of a one-signed tile's magnitudes
+#endif
+#ifndef DAB_PIX_OCTAVES_MIXED_LOG2
+#define DAB_PIX_OCTAVES_MIXED_LOG2 3  // and the top 2^3 = 8 octaves on either side of zero of a tile with both signs
 #endif
 
 template <bool kOctaves>
@@ -104,9 +107,11 @@ __device__ __forceinline__ PixQuant make_pix_quant(uint32_t kmin, uint32_t kmax,
   q.B0 = lo > 0.0f ? 0 : (hi < 0.0f ? (1 << LOG2B) : (1 << (LOG2B - 1)));
   q.shift = 0;
   q.p = (kc + 127) << 23;
-  if (kOctaves && !mixed) {  // 2^m buckets per octave; e >= -40 keeps the base positive
-    q.shift = 23 - (LOG2B - DAB_PIX_OCTAVES_LOG2);
-    q.p = (int)(__float_as_uint(A) >> q.shift) - ((1 << LOG2B) - 1);
+  if (kOctaves) {  // 2^m buckets per octave; e >= -40 keeps the base positive
+    // one sign: all B buckets over the top four octaves; both signs: B/2 per sign over the top eight
+    const int side = mixed ? (1 << (LOG2B - 1)) : (1 << LOG2B);
+    q.shift = 23 - (mixed ? LOG2B - 1 - DAB_PIX_OCTAVES_MIXED_LOG2 : LOG2B - DAB_PIX_OCTAVES_LOG2);
+    q.p = (int)(__float_as_uint(A) >> q.shift) - (side - 1);
   }
   return q;
 }
@@ -114,9 +119,10 @@ __device__ __forceinline__ PixQuant make_pix_quant(uint32_t kmin, uint32_t kmax,
 // (A negative value so small that the product rounds to -0.0 still belongs below zero.)
 template <bool kOctaves>
 __device__ __forceinline__ int pix_bucket(float v, const PixQuant& q, int B) {
-  if (kOctaves && q.shift) {  // one sign only: magnitudes ascend with the bucket for positive tiles, descend for negative ones
-    const int i = min(max((int)((__float_as_uint(v) & 0x7FFFFFFFu) >> q.shift) - q.p, 0), B - 1);
-    return q.B0 ? B - 1 - i : i;
+  if (kOctaves && q.shift) {  // magnitudes ascend with the bucket on the positive side, descend on the negative one
+    const int side = (q.B0 > 0 && q.B0 < B) ? B >> 1 : B;  // buckets per sign
+    const int i = min(max((int)((__float_as_uint(v) & 0x7FFFFFFFu) >> q.shift) - q.p, 0), side - 1);
+    return v < 0.0f ? q.B0 - 1 - i : q.B0 + i;
   }
   int f = __float2int_rd(v * __int_as_float(q.p));
   if (v < 0.0f) f = min(f, -1);
@@ -129,11 +135,12 @@ template <bool kOctaves>
 __device__ __forceinline__ void pix_bucket_range(const PixQuant& q, int b, int B, double& vlo, double& vhi,
                                                  double& inv_width) {
   if (kOctaves && q.shift) {
-    const int i = q.B0 ? B - 1 - b : b;
+    const bool negative = b < q.B0;
+    const int i = negative ? q.B0 - 1 - b : b - q.B0;
     const float lo = i ? __uint_as_float((uint32_t)(i + q.p) << q.shift) : 0.0f;
     const float hi = __uint_as_float((uint32_t)(i + 1 + q.p) << q.shift);
-    vlo = q.B0 ? -(double)hi : (double)lo;
-    vhi = q.B0 ? -(double)lo : (double)hi;
+    vlo = negative ? -(double)hi : (double)lo;
+    vhi = negative ? -(double)lo : (double)hi;
     // hi - lo = 2^(exponent of lo - m) with m = 23 - shift: its reciprocal by exponent arithmetic; next to zero 1 / hi
     const int biased = (int)((uint32_t)(i + q.p) >> (23 - q.shift));  // exponent field of lo
     const double r = i ? (double)__int_as_float((254 + (23 - q.shift) - biased) << 23) : (double)__fdividef(1.0f, hi);
@@ -226,18 +233,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
   ListT* list = reinterpret_cast<ListT*>(off + (KHW ? 0 : ((a.n + 1) & ~1)));  // [pix][C] channels by bucket
 
   __shared__ uint32_t s_kmin, s_kmax;
-  if (a.marked_only) {
-    // the second kernel of a call usually has nothing to do: every thread looks at the first patch of another of
-    // the CTA's tiles, and the CTA leaves before any set-up unless one of them carries the mark
-    const int64_t per_img = (int64_t)a.tiles_h * a.tiles_w, tiles = per_img * a.d.N;
-    int any = 0;
-    for (int64_t t = blockIdx.x + (int64_t)threadIdx.x * gridDim.x; t < tiles; t += (int64_t)THREADS * gridDim.x) {
-      const int img = (int)(t / per_img), trem = (int)(t % per_img);
-      const int64_t first = ((int64_t)img * a.Ho + (trem / a.tiles_w) * a.TH) * a.Wo + (trem % a.tiles_w) * a.TW;
-      any |= a.pK[DAB_IDX(first, patch_count(a))] == kRowMark;
-    }
-    if (!__syncthreads_or(any)) return;
-  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int C = a.d.C, pixn = a.pix, chw = a.ch_words, khw = a.d.kh * a.d.kw;
   uint32_t* scratch = scratch_all + warp * kHullCap;
@@ -273,7 +268,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     const int th = min(a.TH, a.Ho - ho0), tw = min(a.TW, a.Wo - wo0);
     const int npatch = th * tw;
     const int64_t tile_base = ((int64_t)img * a.Ho + ho0) * a.Wo + wo0;  // index of the tile's first patch
-    if (a.marked_only && a.pK[DAB_IDX(tile_base, patch_count(a))] != kRowMark) continue;  // the same for every thread
     __syncthreads();  // the previous tile is no longer read
     if (threadIdx.x == 0) { s_kmin = kPadKey; s_kmax = 0u; }
     for (int i = threadIdx.x; i < pixn * SS; i += THREADS) { cntc[i] = 0; sumc[i] = 0.0; }
@@ -328,9 +322,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) binarize_patches_pixhist_ker
     const uint32_t tkmin = s_kmin, tkmax = s_kmax;
     const bool any_nonzero = tkmin <= tkmax;
     PixQuant qz = make_pix_quant<kOctaves>(any_nonzero ? tkmin : kZeroKey + 1u, any_nonzero ? tkmax : kZeroKey + 1u, LOG2B);
-    const bool both_signs = any_nonzero && key_value(tkmin) < 0.0f && key_value(tkmax) > 0.0f;
-    if (any_nonzero && (key_range_nonfinite(tkmin, tkmax) || !qz.ok || (a.defer_mixed && both_signs))) {
-      // every patch of the tile is left to the next kernel of the call
+    if (any_nonzero && (key_range_nonfinite(tkmin, tkmax) || !qz.ok)) {
+      // every patch of the tile is left to the sorting kernel
       for (int p = threadIdx.x; p < npatch; p += THREADS) {
         const int64_t pi = tile_base + (int64_t)(p / tw) * a.Wo + p % tw;
         if (DAB_IN_BOUNDS(pi, patch_count(a))) a.pK[pi] = kRowMark;
@@ -860,30 +853,13 @@ cudaError_t launch_binarize_patches_pixhist(const dab_conv_desc& d, int32_t Ho, 
   *applicable = false;
   if (a.n <= 256 || a.n > 8192 || d.kh * d.kw > 64) return cudaSuccess;
   cudaError_t e;
-  // Buckets by patch length.  Tiles of one sign (post-ReLU activations) take the per-octave grid, under which 32
-  // buckets leave a hull of about 17 values of a row of 576 and of about 36 of a row of 1152; the first kernel is
-  // sized for them.  A tile with both signs needs the equal-width grid with twice the buckets: rows of 1024 values
-  // and more leave such tiles (all their patches marked) to a second kernel with twice the buckets per lane, which
-  // looks at the first patch of every tile and codes the marked tiles only.
-  a.defer_mixed = a.n >= DAB_PIX_N1 ? 1 : 0;
-  a.marked_only = 0;
-  PixArgs second = a;
-  second.defer_mixed = 0;
-  second.marked_only = 1;
-  bool second_fits = false;
-  if (a.n < DAB_PIX_N1) {
-    e = launch_pix_for<1>(a, stream, applicable);
-  } else if (a.n < DAB_PIX_N2) {
-    e = launch_pix_for<1>(a, stream, applicable);
-    if (e == cudaSuccess && *applicable) e = launch_pix_for<2>(second, stream, &second_fits);
-  } else if (a.n < DAB_PIX_N4) {
-    e = launch_pix_for<2>(a, stream, applicable);
-    if (e == cudaSuccess && *applicable) e = launch_pix_for<4>(second, stream, &second_fits);
-  } else {
-    e = launch_pix_for<4>(a, stream, applicable);
-    if (e == cudaSuccess && *applicable) e = launch_pix_for<8>(second, stream, &second_fits);
-  }
-  // (a second kernel that fits no tile launches nothing: the marked tiles then go to the sorting kernel below)
+  // Buckets by patch length: 32 below 2048 values, 64 below 4096, 128 beyond.  Under the per-octave grids that
+  // leaves a hull of about 17 values of a post-ReLU row of 576 and about 36 of a row of 1152 (with twice the buckets
+  // the smaller hull saves less than tables, assembly and bounds cost; with equal-width buckets the hulls were three
+  // times as long with the same number of buckets).
+  if (a.n < DAB_PIX_N2) e = launch_pix_for<1>(a, stream, applicable);
+  else if (a.n < DAB_PIX_N4) e = launch_pix_for<2>(a, stream, applicable);
+  else e = launch_pix_for<4>(a, stream, applicable);
   if (e != cudaSuccess || !*applicable) return e;
   if (a.n <= 2048) return launch_fixup<8>(a, stream);
   if (a.n <= 4096) return launch_fixup<16>(a, stream);
